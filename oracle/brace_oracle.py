@@ -1,0 +1,361 @@
+"""CPU oracle for BRACE ring aggregation.  TEST INFRASTRUCTURE ONLY.
+
+This module is a plain, slow, by-eye-checkable numpy restatement of what the
+paper "Byzantine-Robust Federated Learning over Ring-All-Reduce Distributed
+Computing" (BRACE) computes in one aggregation round.  It exists to check the
+CUDA library; it is never part of the product path.  Only the test-suite, the
+smoke check and the benchmark's CPU-baseline / reference legs may import it.
+It shares no code with the CUDA library and imports nothing from it.
+
+Every function names the passage of the paper it follows.  Where the method
+has an exact plain definition (Eq. (1): a threshold on an integer sum) the
+oracle is that definition; where the paper describes a procedure (the ring
+schedule of Section 2.2 and Section 3) the oracle performs the procedure hop
+by hop on literal per-client arrays, snapshotting every message of a hop
+before applying any of them, exactly as n concurrent clients would.
+
+Readings of points the paper leaves open (all are parameters, defaults below):
+  * sign(0) = 0, sign(NaN) = 0, sign(+-Inf) = +-1 (``zero_sign`` in {-1,0,+1}
+    maps exact zeros elsewhere); Section 3 Phase I only says "element-wise sign".
+  * lambda may be any finite real; the sign-sum is an integer, so
+    ``S > lambda`` is evaluated as ``S > floor(lambda)``; ties give -1 as
+    Eq. (1) prints.
+  * "n roughly equal-sized sub-vectors" (Section 2.2): sub-vector boundaries
+    fall on multiples of a granule of G coordinates, see ``partition``.
+  * ring direction and hop -> sub-vector map: fixed by the three-client worked
+    example of Section 2.2 (0-based: at share-reduce hop s client c sends
+    sub-vector (c - s) mod n to client (c + 1) mod n; after n-1 hops client c
+    owns sub-vector (c + 1) mod n; at share-only hop t client c sends
+    sub-vector (c + 1 - t) mod n).
+
+Parity status: every function here is pinned by tests/test_oracle_pins.py
+(printed worked example, closed forms, invariants, brute force); none is
+"parity unpinned".
+"""
+
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+
+RULE_SIGN_CONSENSUS = 0  # BRACE, Section 3, Eq. (1)
+RULE_SUM = 1             # plain ring-all-reduce, Section 2.2
+
+ATTACK_SCALE_OWN = 1     # b_i = a * h_i
+ATTACK_GAUSSIAN = 2      # b_i = sigma * z_i
+ATTACK_SCALED_MEAN = 3   # b_i = a * mean_honest
+ATTACK_MEAN_SHIFT = 4    # b_i = mean_honest - kappa * std_honest
+ATTACK_SPARSE_NOISE = 5  # b_i[k] = sigma * z_i[k] if u_i[k] < p else 0
+
+
+# --------------------------------------------------------------------------
+# Section 2.2: "splitting its gradient into n roughly equal-sized sub-vectors"
+# --------------------------------------------------------------------------
+def partition(n: int, d: int, granule: int = 128):
+    """Sub-vector j covers coordinates [begin_j, end_j).
+
+    The d coordinates are grouped into Q = ceil(d / G) granules of G
+    coordinates (the last one possibly short); sub-vector j takes granules
+    floor(j*Q/n) .. floor((j+1)*Q/n) - 1.  G = 1 is the balanced split of d
+    into n parts.  Sub-vectors may be empty when d < n*G.
+    """
+    if n < 2 or d < 1 or granule < 1:
+        raise ValueError("need n >= 2, d >= 1, granule >= 1")
+    q = -(-d // granule)
+    bounds = []
+    for j in range(n):
+        b = min(granule * ((j * q) // n), d)
+        e = min(granule * (((j + 1) * q) // n), d)
+        bounds.append((b, e))
+    return bounds
+
+
+# --------------------------------------------------------------------------
+# Section 3, Phase I (Quantization): element-wise sign
+# --------------------------------------------------------------------------
+def sgn(x: np.ndarray, zero_sign: int = 0) -> np.ndarray:
+    """Element-wise sign as int32: (x > 0) - (x < 0); exact zeros and NaN give
+    ``zero_sign`` for zeros and 0 for NaN."""
+    x = np.asarray(x)
+    s = (x > 0).astype(np.int32) - (x < 0).astype(np.int32)
+    if zero_sign != 0:
+        s = np.where(x == 0, np.int32(zero_sign), s)
+    return s.astype(np.int32)
+
+
+def lambda_int(lam: float, n: int) -> int:
+    """Integer threshold equivalent to the real lambda of Eq. (1): for integer S,
+    S > lambda  <=>  S > floor(lambda); clamped to [-n-1, n] (beyond that range
+    the comparison is constant)."""
+    if not math.isfinite(lam):
+        raise ValueError("lambda must be finite")
+    return int(max(-n - 1, min(n, math.floor(lam))))
+
+
+# --------------------------------------------------------------------------
+# Section 3, Phase III, Eq. (1): the aggregation rule as a plain definition
+# --------------------------------------------------------------------------
+def gar_direct(updates: np.ndarray, lam: float, zero_sign: int = 0) -> np.ndarray:
+    """GAR(g_1..g_n)[k] = +1 if sum_i sign(g_i[k]) > lambda else -1 (Eq. (1)).
+
+    updates: [n, d].  Returns int8 [d] with entries in {-1, +1}.
+    """
+    updates = np.asarray(updates)
+    n = updates.shape[0]
+    total = np.zeros(updates.shape[1], dtype=np.int32)
+    for i in range(n):
+        total = total + sgn(updates[i], zero_sign)
+    lam_i = lambda_int(lam, n)
+    return np.where(total > lam_i, 1, -1).astype(np.int8)
+
+
+def sign_sum_direct(updates: np.ndarray, zero_sign: int = 0) -> np.ndarray:
+    """S[k] = sum_i sign(g_i[k]) (the quantity thresholded in Eq. (1))."""
+    updates = np.asarray(updates)
+    total = np.zeros(updates.shape[1], dtype=np.int32)
+    for i in range(updates.shape[0]):
+        total = total + sgn(updates[i], zero_sign)
+    return total
+
+
+# --------------------------------------------------------------------------
+# Output representation: 1 bit per dimension (Section 3, cost paragraph)
+# --------------------------------------------------------------------------
+def pack_bits(pm1: np.ndarray, words: int | None = None) -> np.ndarray:
+    """Pack a {-1,+1} vector into uint32 words: coordinate k is bit (k mod 32),
+    least significant first, of word (k div 32); +1 -> 1, -1 -> 0; padding 0."""
+    pm1 = np.asarray(pm1)
+    d = pm1.shape[0]
+    nwords = -(-d // 32) if words is None else words
+    out = np.zeros(nwords, dtype=np.uint32)
+    for k in range(d):
+        if pm1[k] > 0:
+            out[k // 32] |= np.uint32(1) << np.uint32(k % 32)
+    return out
+
+
+def pack_bits_fast(pm1: np.ndarray, words: int | None = None) -> np.ndarray:
+    """Same mapping as ``pack_bits`` through numpy's packbits (little bit order);
+    tests check the two agree."""
+    pm1 = np.asarray(pm1)
+    d = pm1.shape[0]
+    nwords = -(-d // 32) if words is None else words
+    bits = np.zeros(nwords * 32, dtype=np.uint8)
+    bits[:d] = pm1 > 0
+    return np.packbits(bits, bitorder="little").view("<u4").astype(np.uint32)
+
+
+# --------------------------------------------------------------------------
+# Sections 2.2 and 3: the ring procedure, hop by hop
+# --------------------------------------------------------------------------
+@dataclass
+class RingTrace:
+    """Everything a round of the ring leaves behind.
+
+    outputs      [n, d]  what each client holds after Share-Only
+                         (int8 +-1 for BRACE, float32 for SUM)
+    rs_states    list over share-reduce hops s of a list over clients r of
+                 (sub-vector id, copy of client r's reduced partial for that
+                 sub-vector after hop s)
+    owned        list over clients c of (sub-vector id, fully reduced partial)
+                 after the last share-reduce hop
+    rs_sent      [n] coordinates each client sent during share-reduce
+    ag_sent      [n] coordinates each client sent during share-only
+    bounds       the partition used
+    """
+    outputs: np.ndarray
+    rs_states: list = field(default_factory=list)
+    owned: list = field(default_factory=list)
+    rs_sent: np.ndarray | None = None
+    ag_sent: np.ndarray | None = None
+    bounds: list = field(default_factory=list)
+    ag_states: list = field(default_factory=list)
+
+
+def ring_round(updates: np.ndarray, rule: int = RULE_SIGN_CONSENSUS, lam: float = 0.0,
+               zero_sign: int = 0, granule: int = 128, mean: bool = False,
+               keep_states: bool = True) -> RingTrace:
+    """One aggregation round on literal per-client arrays.
+
+    BRACE (rule = RULE_SIGN_CONSENSUS), Section 3:
+      Phase I   every client replaces its vector by its element-wise sign;
+      Phase II  share-reduce: n-1 hops; at hop s client c sends its current
+                sub-vector (c - s) mod n downstream, the receiver adds it to its
+                own copy of that sub-vector;
+      Phase III the owner of each fully reduced sub-vector thresholds it with
+                lambda (Eq. (1));
+      Phase IV  share-only: n-1 hops; at hop t client c sends sub-vector
+                (c + 1 - t) mod n downstream, the receiver overwrites.
+    Plain RAR (rule = RULE_SUM), Section 2.2: same Phases II and IV on the raw
+    float32 vectors (additions in float32, in the order the ring performs
+    them); Phase III is the identity, or division by n when ``mean`` is set.
+    """
+    updates = np.asarray(updates)
+    n, d = updates.shape
+    bounds = partition(n, d, granule)
+
+    # Phase I (BRACE) / local copies (SUM): one full-length working vector per client
+    if rule == RULE_SIGN_CONSENSUS:
+        work = [sgn(updates[c], zero_sign) for c in range(n)]
+    elif rule == RULE_SUM:
+        work = [np.array(updates[c], dtype=np.float32, copy=True) for c in range(n)]
+    else:
+        raise ValueError("unknown rule")
+
+    trace = RingTrace(outputs=np.empty(0), bounds=bounds)
+    rs_sent = np.zeros(n, dtype=np.int64)
+    ag_sent = np.zeros(n, dtype=np.int64)
+
+    # Phase II: Share-Reduce
+    for s in range(n - 1):
+        messages = []
+        for c in range(n):                      # all clients send at once: snapshot first
+            j = (c - s) % n
+            b, e = bounds[j]
+            messages.append((c, j, work[c][b:e].copy()))
+            rs_sent[c] += e - b
+        states = []
+        for c, j, payload in messages:          # then every receiver reduces
+            r = (c + 1) % n
+            b, e = bounds[j]
+            work[r][b:e] = payload + work[r][b:e]
+        if keep_states:
+            for r in range(n):
+                j = (r - 1 - s) % n
+                b, e = bounds[j]
+                states.append((j, work[r][b:e].copy()))
+            trace.rs_states.append(states)
+
+    # ownership after n-1 hops: client c holds the reduced sub-vector (c+1) mod n
+    for c in range(n):
+        j = (c + 1) % n
+        b, e = bounds[j]
+        trace.owned.append((j, work[c][b:e].copy()))
+
+    # Phase III: Consensus (BRACE) / identity or mean (SUM), local to the owner
+    if rule == RULE_SIGN_CONSENSUS:
+        lam_i = lambda_int(lam, n)
+        result = [np.zeros(d, dtype=np.int8) for _ in range(n)]
+        for c in range(n):
+            j = (c + 1) % n
+            b, e = bounds[j]
+            result[c][b:e] = np.where(work[c][b:e] > lam_i, 1, -1).astype(np.int8)
+    else:
+        result = [np.zeros(d, dtype=np.float32) for _ in range(n)]
+        for c in range(n):
+            j = (c + 1) % n
+            b, e = bounds[j]
+            seg = work[c][b:e]
+            result[c][b:e] = (seg / np.float32(n)) if mean else seg
+
+    # Phase IV: Share-Only
+    for t in range(n - 1):
+        messages = []
+        for c in range(n):
+            j = (c + 1 - t) % n
+            b, e = bounds[j]
+            messages.append((c, j, result[c][b:e].copy()))
+            ag_sent[c] += e - b
+        for c, j, payload in messages:
+            r = (c + 1) % n
+            b, e = bounds[j]
+            result[r][b:e] = payload
+        if keep_states:
+            trace.ag_states.append([row.copy() for row in result])
+
+    trace.outputs = np.stack(result)
+    trace.rs_sent = rs_sent
+    trace.ag_sent = ag_sent
+    return trace
+
+
+def sum_direct_f64(updates: np.ndarray) -> np.ndarray:
+    """sum_i g_i in float64 (Section 2.2: what every client holds after RAR)."""
+    updates = np.asarray(updates)
+    acc = np.zeros(updates.shape[1], dtype=np.float64)
+    for i in range(updates.shape[0]):
+        acc = acc + updates[i].astype(np.float64)
+    return acc
+
+
+# --------------------------------------------------------------------------
+# Section 2.2 / Section 3 / Table 1: bits each client sends per round
+# --------------------------------------------------------------------------
+def sent_bits(trace: RingTrace, m_bits: int, rule: int) -> np.ndarray:
+    """Bits sent per client: share-reduce moves m bits per coordinate; share-only
+    moves 1 bit per coordinate under BRACE and m bits under plain RAR."""
+    ag_width = 1 if rule == RULE_SIGN_CONSENSUS else m_bits
+    return trace.rs_sent * m_bits + trace.ag_sent * ag_width
+
+
+def cost_sc(m, n, d):      # Section 2.2, Table 1
+    return m * n * d
+
+
+def cost_rar(m, n, d):     # Section 2.2, Table 1 (exact rational kept as a pair)
+    return 2 * m * d * (n - 1), n
+
+
+def cost_brace(m, n, d):   # Section 3, Table 1
+    return d * (n - 1) * (m + 1), n
+
+
+# --------------------------------------------------------------------------
+# Section 3 (threat model): Byzantine clients alter their vectors before the
+# ring starts.  The five synthetic alterations of the benchmark workloads.
+# --------------------------------------------------------------------------
+def inject_attack(kind: int, honest: np.ndarray, byz_ids, *, scale: float = 1.0,
+                  sigma: float = 1.0, kappa: float = 3.0, prob: float = 0.1,
+                  noise: np.ndarray | None = None,
+                  uniform: np.ndarray | None = None) -> np.ndarray:
+    """Return the update matrix the ring will see: honest rows unchanged,
+    Byzantine rows replaced.  Arithmetic in float64, one final rounding to
+    float32.  ``noise`` / ``uniform`` are [len(byz_ids), d] arrays of standard
+    normal / uniform[0,1) draws supplied by the caller (row b belongs to
+    byz_ids[b]).  Statistics over honest rows accumulate in increasing client id.
+    """
+    honest = np.asarray(honest, dtype=np.float32)
+    n, d = honest.shape
+    byz_ids = [int(i) for i in byz_ids]
+    byz = set(byz_ids)
+    good = [i for i in range(n) if i not in byz]
+    out = honest.copy()
+    if not byz_ids:
+        return out
+
+    if kind == ATTACK_SCALE_OWN:
+        for i in byz_ids:
+            out[i] = (np.float64(np.float32(scale)) * honest[i].astype(np.float64)).astype(np.float32)
+    elif kind == ATTACK_GAUSSIAN:
+        for b, i in enumerate(byz_ids):
+            out[i] = (np.float64(np.float32(sigma)) * noise[b].astype(np.float64)).astype(np.float32)
+    elif kind in (ATTACK_SCALED_MEAN, ATTACK_MEAN_SHIFT):
+        m = len(good)
+        if m == 0:
+            raise ValueError("no honest client to take statistics over")
+        total = np.zeros(d, dtype=np.float64)
+        for i in good:
+            total = total + honest[i].astype(np.float64)
+        mean = total / np.float64(m)
+        if kind == ATTACK_SCALED_MEAN:
+            vec = np.float64(np.float32(scale)) * mean
+        else:
+            sq = np.zeros(d, dtype=np.float64)
+            for i in good:
+                dev = honest[i].astype(np.float64) - mean
+                sq = sq + dev * dev
+            std = np.sqrt(sq / np.float64(m))          # population std (ddof = 0)
+            vec = mean - np.float64(np.float32(kappa)) * std
+        vec32 = vec.astype(np.float32)
+        for i in byz_ids:
+            out[i] = vec32
+    elif kind == ATTACK_SPARSE_NOISE:
+        p32 = np.float32(prob)
+        for b, i in enumerate(byz_ids):
+            val = (np.float64(np.float32(sigma)) * noise[b].astype(np.float64)).astype(np.float32)
+            out[i] = np.where(uniform[b].astype(np.float32) < p32, val, np.float32(0.0))
+    else:
+        raise ValueError("unknown attack kind")
+    return out
