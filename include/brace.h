@@ -1,0 +1,225 @@
+/*
+ * brace.h -- C ABI of the BRACE ring-aggregation library for NVIDIA B200 (sm_100a).
+ *
+ * One aggregation round of "Byzantine-Robust Federated Learning over
+ * Ring-All-Reduce Distributed Computing" (BRACE): n clients each hold an update
+ * vector of d float32 coordinates; the round leaves every client with the same
+ * aggregated vector.  The n clients and the ring between them are simulated on
+ * one GPU: client c's data are row c of caller-owned device matrices, a hop is
+ * a move of one sub-vector from row c's buffers into row (c+1) mod n's.
+ *
+ * Conventions shared by every call
+ *   - returns an int status (BRACE_OK = 0); never throws, aborts or prints;
+ *   - device work is enqueued on `stream` (a cudaStream_t passed as void*) and
+ *     the call returns without synchronising;
+ *   - the library allocates no device memory: mailboxes live in the
+ *     caller-provided workspace, inputs and outputs are caller buffers;
+ *   - pointers named d_* are device pointers, h_* host pointers;
+ *   - clients c and sub-vectors j are 0-based.  Ring direction and the
+ *     hop -> sub-vector map follow the three-client worked example of
+ *     Section 2.2: at share-reduce hop s client c sends sub-vector
+ *     (c - s) mod n to client (c + 1) mod n; after n-1 hops client c owns
+ *     sub-vector (c + 1) mod n; at share-only hop t client c sends
+ *     sub-vector (c + 1 - t) mod n to client (c + 1) mod n.
+ *   - a context must not be used from two host threads, or on two streams,
+ *     at the same time.
+ */
+#ifndef BRACE_H
+#define BRACE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct brace_ctx brace_ctx;
+typedef void* brace_stream_t; /* cudaStream_t */
+
+/* status codes */
+enum {
+  BRACE_OK = 0,
+  BRACE_ERR_INVALID_ARG = 1, /* null / out-of-range / misaligned argument; nothing was launched */
+  BRACE_ERR_UNSUPPORTED = 2, /* valid request this build cannot serve (e.g. n > 32767)          */
+  BRACE_ERR_BAD_STEP = 3,    /* hop called out of order; nothing was launched                   */
+  BRACE_ERR_WORKSPACE = 4,   /* workspace missing, too small or misaligned                      */
+  BRACE_ERR_CUDA = 5,        /* a CUDA runtime call failed; see brace_last_cuda_error           */
+  BRACE_ERR_TIMEOUT = 6      /* reserved: a bounded device-side wait ran out                    */
+};
+
+/* aggregation rules */
+enum {
+  BRACE_RULE_SIGN_CONSENSUS = 0, /* BRACE, Section 3, Eq. (1)                                     */
+  BRACE_RULE_SUM = 1             /* plain ring-all-reduce sum, Section 2.2 (optionally the mean)  */
+};
+
+/* how brace_aggregate runs a round (the result is the same) */
+enum {
+  BRACE_AGG_AUTO = 0,     /* fused when the layout allows it, else stepwise                        */
+  BRACE_AGG_STEPWISE = 1, /* 2(n-1)+1 kernel launches, one per hop, exactly like the step calls    */
+  BRACE_AGG_FUSED = 2     /* one kernel that carries each sub-vector tile through all hops         */
+};
+
+/* Byzantine alterations applied before the ring starts (threat model, Section 3).
+ * "honest" rows are those not listed as Byzantine; statistics over them are
+ * accumulated in float64 in increasing client id and rounded once to float32. */
+enum {
+  BRACE_ATTACK_NONE = 0,
+  BRACE_ATTACK_SCALE_OWN = 1,   /* b_i = scale * h_i (own honest update)                           */
+  BRACE_ATTACK_GAUSSIAN = 2,    /* b_i = sigma * noise_i                                           */
+  BRACE_ATTACK_SCALED_MEAN = 3, /* b_i = scale * mean_honest (same vector for every Byzantine)     */
+  BRACE_ATTACK_MEAN_SHIFT = 4,  /* b_i = mean_honest - kappa * std_honest (population std)         */
+  BRACE_ATTACK_SPARSE_NOISE = 5 /* b_i[k] = uniform_i[k] < prob ? sigma * noise_i[k] : 0           */
+};
+
+/* Parameters of the rule.  Fill with brace_default_params, then edit. */
+typedef struct brace_params {
+  int32_t rule;      /* BRACE_RULE_*                                                              */
+  float lambda;      /* Eq. (1) threshold; any finite value; the sign-sum S is an integer, so
+                        S > lambda is evaluated as S > floor(lambda); S == lambda gives -1        */
+  int32_t zero_sign; /* what an exactly-zero coordinate votes: -1, 0 (default, abstain) or +1;
+                        NaN always votes 0, +-Inf vote +-1                                        */
+  int32_t granule;   /* sub-vector boundaries are multiples of this many coordinates
+                        (default 128; >= 1).  With Q = ceil(d/granule), sub-vector j is
+                        [min(granule*floor(j*Q/n), d), min(granule*floor((j+1)*Q/n), d))          */
+  int32_t mean;      /* BRACE_RULE_SUM only: non-zero divides the sum by n                        */
+  int32_t agg_mode;  /* BRACE_AGG_*                                                               */
+} brace_params;
+
+/* Description of one attack.  noise / uniform are [f][*_ld] float32 matrices of
+ * standard-normal / uniform[0,1) draws supplied by the caller (row b belongs to
+ * the b-th Byzantine id); only the kinds that consume them read them. */
+typedef struct brace_attack {
+  int32_t kind;             /* BRACE_ATTACK_*                                                     */
+  float scale;              /* kinds 1, 3                                                         */
+  float sigma;              /* kinds 2, 5                                                         */
+  float kappa;              /* kind 4                                                             */
+  float prob;               /* kind 5                                                             */
+  const int32_t* h_byz_ids; /* host array of f distinct client ids, or NULL for clients 0..f-1    */
+  const float* noise;       /* device pointer (host pointer for brace_aggregate_host)             */
+  int64_t noise_ld;
+  const float* uniform;     /* device pointer (host pointer for brace_aggregate_host)             */
+  int64_t uniform_ld;
+} brace_attack;
+
+const char* brace_status_string(int status);
+
+/* rule = SIGN_CONSENSUS, lambda = 0, zero_sign = 0, granule = 128, mean = 0, agg_mode = AUTO. */
+int brace_default_params(brace_params* params);
+
+/* Bytes of device workspace a context for (n, d, params) needs; 0 if the
+ * arguments are invalid.  Holds two sets ("ping-pong") of n mailboxes, each as
+ * long as the longest sub-vector rounded up to 128 entries, plus client-id
+ * lists for the attack kernels.  Mailbox entries are int8 partial sign-sums
+ * for n <= 127, int16 for n <= 32767 (BRACE), float32 (SUM). */
+size_t brace_workspace_bytes(int32_t n, int64_t d, const brace_params* params);
+
+/* Create a context (host memory, owned by the library until brace_destroy).
+ *   n >= 2 clients, 0 <= f < n of them Byzantine (f is used by the attack call
+ *   and by validation only -- Eq. (1) does not take f), d >= 1 coordinates.
+ *   d_workspace: device memory, 256-byte aligned, at least brace_workspace_bytes
+ *   long, owned by the caller and kept alive and untouched while the context
+ *   lives.  Passing d_workspace = NULL with workspace_bytes = 0 creates a
+ *   host-only context: brace_segment works, every device call returns
+ *   BRACE_ERR_WORKSPACE.  `stream` is accepted for symmetry; init enqueues nothing.
+ * Errors: INVALID_ARG (null out, n < 2, f out of range, d < 1, bad params,
+ * non-finite lambda), UNSUPPORTED (n > 32767 under SIGN_CONSENSUS),
+ * WORKSPACE (too small / misaligned). */
+int brace_init(brace_ctx** out, int32_t n, int32_t f, int64_t d, const brace_params* params,
+               void* d_workspace, size_t workspace_bytes, brace_stream_t stream);
+int brace_destroy(brace_ctx* ctx);
+
+/* Sub-vector j covers coordinates [*begin, *end) (Section 2.2: "n roughly
+ * equal-sized sub-vectors"; formula at brace_params.granule).  Host only. */
+int brace_segment(const brace_ctx* ctx, int32_t j, int64_t* begin, int64_t* end);
+
+/* cudaError_t of the last failed runtime call on this context (0 if none). */
+int brace_last_cuda_error(const brace_ctx* ctx);
+
+/* Threat model of Section 3: Byzantine clients alter their vectors before the
+ * ring starts and then follow the protocol.  Reads the honest update matrix
+ * d_honest [n][ld_honest] and writes the f Byzantine rows of d_updates
+ * [n][ld_updates]; rows of honest clients are not touched.  d_honest may equal
+ * d_updates (in place).  attack->noise / uniform are device pointers.
+ * kind NONE or f == 0 does nothing.  Errors: INVALID_ARG (null pointers, ld < d,
+ * duplicate or out-of-range ids, missing noise/uniform for a kind that needs
+ * them). */
+int brace_inject_attack(brace_ctx* ctx, const brace_attack* attack, const float* d_honest,
+                        int64_t ld_honest, float* d_updates, int64_t ld_updates,
+                        brace_stream_t stream);
+
+/* Section 3 Phase I (Quantization) on its own: d_q [n][ld_q] int8 receives the
+ * element-wise sign of d_updates [n][ld].  The ring calls below fuse this step
+ * into their reads; this entry exists for inspection and tests. */
+int brace_quantize(brace_ctx* ctx, const float* d_updates, int64_t ld, int8_t* d_q, int64_t ld_q,
+                   brace_stream_t stream);
+
+/* One Share-Reduce hop (Section 2.2 Phase I / Section 3 Phase II) for all n
+ * clients at once.  Receiver r = (c+1) mod n stores into its mailbox the value
+ * it received from c (c's own quantized sub-vector at step 0, c's mailbox
+ * content otherwise) plus its own (quantized) sub-vector (c - step) mod n.
+ * step must run 0, 1, .., n-2 in order; step 0 may be called at any time and
+ * starts a new round.  d_updates [n][ld] float32, ld >= d, must not change
+ * during a round.  Errors: BAD_STEP, INVALID_ARG, WORKSPACE, CUDA. */
+int brace_ring_reduce_scatter_step(brace_ctx* ctx, int32_t step, const float* d_updates, int64_t ld,
+                                   brace_stream_t stream);
+
+/* Section 3 Phase III (Consensus), after the last share-reduce hop: client c,
+ * owner of sub-vector (c+1) mod n, applies Eq. (1) to the sign-sums in its
+ * mailbox and writes the result into its own output row.
+ *   SIGN_CONSENSUS: d_out is uint32 [n][out_ld], out_ld >= ceil(d/32);
+ *     coordinate k is bit (k mod 32), least significant first, of word
+ *     (k div 32) of the row; 1 means +1, 0 means -1; bits past d in the last
+ *     word are 0.
+ *   SUM: d_out is float32 [n][out_ld], out_ld >= d; the step copies the sum
+ *     (divided by n if params.mean).
+ * Only the owner's sub-vector of each row is written here. */
+int brace_consensus(brace_ctx* ctx, void* d_out, int64_t out_ld, brace_stream_t stream);
+
+/* One Share-Only hop (Section 2.2 Phase II / Section 3 Phase IV) for all n
+ * clients: row (c+1) mod n of d_out receives sub-vector (c + 1 - step) mod n
+ * from row c.  step runs 0..n-2 in order after brace_consensus; after the last
+ * one every row of d_out holds the same aggregated vector. */
+int brace_ring_allgather_step(brace_ctx* ctx, int32_t step, void* d_out, int64_t out_ld,
+                              brace_stream_t stream);
+
+/* A whole round (Section 3, Phases I-IV).  The final contents of every row of
+ * d_out, and of the mailboxes over the lengths of the sub-vectors they hold,
+ * equal those left by calling the step functions in order.  The fused mode needs
+ * granule % 128 == 0, ld % 4 == 0 and 16-byte aligned d_updates (and, for SUM,
+ * out_ld % 4 == 0 and 16-byte aligned d_out); AUTO falls back to stepwise
+ * launches when these do not hold, FUSED returns UNSUPPORTED. */
+int brace_aggregate(brace_ctx* ctx, const float* d_updates, int64_t ld, void* d_out, int64_t out_ld,
+                    brace_stream_t stream);
+
+/* Same round with HOST inputs and outputs: copies h_updates [n][ld] to the
+ * caller's device staging matrix d_updates_stage [n][ld], applies `attack`
+ * there if attack != NULL (attack->noise / uniform are HOST [f][*_ld] matrices,
+ * copied to d_noise_stage / d_uniform_stage of the same shape), aggregates into
+ * d_out_stage [n][out_ld] and copies that to h_out.  All copies are
+ * cudaMemcpyAsync on `stream`: pinned host memory makes them asynchronous, and
+ * h_out is valid once the stream has been synchronised. */
+int brace_aggregate_host(brace_ctx* ctx, const brace_attack* attack, const float* h_updates, int64_t ld,
+                         void* h_out, int64_t out_ld, float* d_updates_stage, float* d_noise_stage,
+                         float* d_uniform_stage, void* d_out_stage, brace_stream_t stream);
+
+/* Test aid: device pointer, length (entries) and sub-vector id of the mailbox
+ * that client `client` filled at the most recent share-reduce hop
+ * (hops_back = 0) or at the hop before it (hops_back = 1; the other mailbox
+ * set).  Valid after at least 1 + hops_back hops of the current round.
+ * *entry_bytes is 1, 2 or 4.  segment and entry_bytes may be NULL. */
+int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back, const void** d_ptr,
+                        int64_t* len, int32_t* segment, int32_t* entry_bytes);
+
+/* Expert knob for measurements: pick the fused kernel's shape.  fused_variant
+ * 0 = library default, 1..5 = (float4 per thread per client, clients
+ * prefetched) in {(1,8),(2,4),(1,4),(2,8),(1,16)}; fused_grid = 0 launches one
+ * CTA per tile, > 0 caps the grid (CTAs then loop over tiles).  Results do not
+ * depend on either. */
+int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BRACE_H */

@@ -1,0 +1,630 @@
+// Host side of the BRACE ring-aggregation library: context, argument checks,
+// the ring-schedule driver and kernel launches.  C ABI declared in brace.h.
+#include "brace.h"
+
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "brace_kernels.cuh"
+
+using namespace brace;
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int64_t kMailAlign = 128;   // mailbox length granularity (entries)
+constexpr int kSmCount = 148;
+
+enum Phase { kIdle = 0, kReducing = 1, kReduced = 2, kConsensusDone = 3, kGathering = 4, kDone = 5 };
+
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+struct brace_ctx {
+  int n = 0, f = 0;
+  int64_t d = 0;
+  brace_params p{};
+  Part pt{};
+  int lam_i = 0;
+  int entry_bytes = 1;
+  int64_t seg_max = 0, seg_pad = 0;
+  char* ws = nullptr;
+  size_t ws_bytes = 0;
+  char* mail[2] = {nullptr, nullptr};
+  int* d_ids = nullptr;
+  // schedule state
+  int phase = kIdle;
+  int rs_done = 0;   // share-reduce hops completed in the current round
+  int ag_done = 0;   // share-only hops completed in the current round
+  int last_cuda = 0;
+  // ids currently stored in d_ids (Byzantine first, then honest), and their staging copy
+  std::vector<int> ids_on_device;
+  std::vector<int> ids_staging;
+  // launch tuning (0 = default)
+  int fused_variant = 0;
+  int fused_grid = 0;
+};
+
+namespace {
+
+bool params_ok(const brace_params* p) {
+  if (!p) return false;
+  if (p->rule != BRACE_RULE_SIGN_CONSENSUS && p->rule != BRACE_RULE_SUM) return false;
+  if (!std::isfinite(p->lambda)) return false;
+  if (p->zero_sign < -1 || p->zero_sign > 1) return false;
+  if (p->granule < 1) return false;
+  if (p->agg_mode < BRACE_AGG_AUTO || p->agg_mode > BRACE_AGG_FUSED) return false;
+  return true;
+}
+
+int entry_bytes_for(int n, int rule) {
+  if (rule == BRACE_RULE_SUM) return 4;
+  if (n <= 127) return 1;
+  if (n <= 32767) return 2;
+  return 0;
+}
+
+Part make_part(int n, int64_t d, int64_t G) {
+  Part pt;
+  pt.d = d;
+  pt.G = G;
+  pt.Q = (d + G - 1) / G;
+  pt.n = n;
+  return pt;
+}
+
+int64_t seg_end(const Part& pt, int j) { return j + 1 == pt.n ? pt.d : pt.begin(j + 1); }
+
+int64_t longest_segment(const Part& pt) {
+  int64_t mx = 0;
+  for (int j = 0; j < pt.n; ++j) {
+    int64_t len = seg_end(pt, j) - pt.begin(j);
+    if (len > mx) mx = len;
+  }
+  return mx;
+}
+
+size_t ids_bytes(int n) { return (size_t)round_up((int64_t)n * 4, 256); }
+
+size_t workspace_need(int n, int64_t d, const brace_params* p) {
+  const int eb = entry_bytes_for(n, p->rule);
+  if (eb == 0) return 0;
+  const Part pt = make_part(n, d, p->granule);
+  const int64_t longest = longest_segment(pt);
+  const int64_t pad = round_up(longest > 0 ? longest : 1, kMailAlign);
+  const size_t one_set = (size_t)round_up((int64_t)n * pad * eb, 256);
+  return 2 * one_set + ids_bytes(n);
+}
+
+int cuda_fail(brace_ctx* ctx, cudaError_t err) {
+  ctx->last_cuda = (int)err;
+  return BRACE_ERR_CUDA;
+}
+
+int check_launch(brace_ctx* ctx) {
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return cuda_fail(ctx, err);
+  return BRACE_OK;
+}
+
+inline unsigned tiles(int64_t items, int64_t per_block) {
+  int64_t t = (items + per_block - 1) / per_block;
+  return (unsigned)(t > 0 ? t : 1);
+}
+
+// ---- launches of the per-hop kernels -------------------------------------------------
+
+bool vec_layout_ok(const brace_ctx* ctx, const float* U, int64_t ld) {
+  return (ctx->p.granule % 4 == 0) && (ld % 4 == 0) && aligned16(U);
+}
+
+int launch_rs_step(brace_ctx* ctx, int step, const float* U, int64_t ld, cudaStream_t st) {
+  const int n = ctx->n;
+  const int in_set = step & 1, out_set = (step + 1) & 1;
+  const bool vec = vec_layout_ok(ctx, U, ld);
+  const int64_t per_block = vec ? kThreads * 4 : kThreads;
+  dim3 grid(tiles(ctx->seg_max, per_block), (unsigned)n);
+  const bool zs = ctx->p.zero_sign != 0;
+  const int zsv = ctx->p.zero_sign;
+#define BRACE_RS_SIGN(P, VEC, ZS)                                                                            \
+  rs_step_sign_kernel<P, VEC, ZS><<<grid, kThreads, 0, st>>>(ctx->pt, U, ld, (const P*)ctx->mail[in_set],    \
+                                                             (P*)ctx->mail[out_set], ctx->seg_pad, step, zsv)
+  if (ctx->p.rule == BRACE_RULE_SUM) {
+    if (vec)
+      rs_step_sum_kernel<true><<<grid, kThreads, 0, st>>>(ctx->pt, U, ld, (const float*)ctx->mail[in_set],
+                                                          (float*)ctx->mail[out_set], ctx->seg_pad, step);
+    else
+      rs_step_sum_kernel<false><<<grid, kThreads, 0, st>>>(ctx->pt, U, ld, (const float*)ctx->mail[in_set],
+                                                           (float*)ctx->mail[out_set], ctx->seg_pad, step);
+  } else if (ctx->entry_bytes == 1) {
+    if (vec) { if (zs) BRACE_RS_SIGN(int8_t, true, true); else BRACE_RS_SIGN(int8_t, true, false); }
+    else     { if (zs) BRACE_RS_SIGN(int8_t, false, true); else BRACE_RS_SIGN(int8_t, false, false); }
+  } else {
+    if (vec) { if (zs) BRACE_RS_SIGN(int16_t, true, true); else BRACE_RS_SIGN(int16_t, true, false); }
+    else     { if (zs) BRACE_RS_SIGN(int16_t, false, true); else BRACE_RS_SIGN(int16_t, false, false); }
+  }
+#undef BRACE_RS_SIGN
+  return check_launch(ctx);
+}
+
+int launch_consensus(brace_ctx* ctx, void* out, int64_t out_ld, cudaStream_t st) {
+  const int n = ctx->n;
+  const int set = (n - 1) & 1;   // the last hop n-2 wrote set (n-1)&1
+  if (ctx->p.rule == BRACE_RULE_SUM) {
+    const bool vec = (ctx->p.granule % 4 == 0) && (out_ld % 4 == 0) && aligned16(out);
+    dim3 grid(tiles(ctx->seg_max, vec ? kThreads * 4 : kThreads), (unsigned)n);
+    if (vec)
+      consensus_sum_kernel<true><<<grid, kThreads, 0, st>>>(ctx->pt, (const float*)ctx->mail[set], ctx->seg_pad,
+                                                            (float*)out, out_ld, ctx->p.mean);
+    else
+      consensus_sum_kernel<false><<<grid, kThreads, 0, st>>>(ctx->pt, (const float*)ctx->mail[set], ctx->seg_pad,
+                                                             (float*)out, out_ld, ctx->p.mean);
+  } else {
+    dim3 grid(tiles(ctx->seg_max / 32 + 2, kThreads), (unsigned)n);
+    if (ctx->entry_bytes == 1)
+      consensus_sign_kernel<int8_t><<<grid, kThreads, 0, st>>>(ctx->pt, (const int8_t*)ctx->mail[set], ctx->seg_pad,
+                                                               (uint32_t*)out, out_ld, ctx->lam_i);
+    else
+      consensus_sign_kernel<int16_t><<<grid, kThreads, 0, st>>>(ctx->pt, (const int16_t*)ctx->mail[set],
+                                                                ctx->seg_pad, (uint32_t*)out, out_ld, ctx->lam_i);
+  }
+  return check_launch(ctx);
+}
+
+int launch_ag_step(brace_ctx* ctx, int step, void* out, int64_t out_ld, cudaStream_t st) {
+  const int n = ctx->n;
+  if (ctx->p.rule == BRACE_RULE_SUM) {
+    const bool vec = (ctx->p.granule % 4 == 0) && (out_ld % 4 == 0) && aligned16(out);
+    dim3 grid(tiles(ctx->seg_max, vec ? kThreads * 4 : kThreads), (unsigned)n);
+    if (vec)
+      ag_step_f32_kernel<true><<<grid, kThreads, 0, st>>>(ctx->pt, (float*)out, out_ld, step);
+    else
+      ag_step_f32_kernel<false><<<grid, kThreads, 0, st>>>(ctx->pt, (float*)out, out_ld, step);
+  } else {
+    dim3 grid(tiles(ctx->seg_max / 32 + 2, kThreads), (unsigned)n);
+    ag_step_bits_kernel<<<grid, kThreads, 0, st>>>(ctx->pt, (uint32_t*)out, out_ld, step);
+  }
+  return check_launch(ctx);
+}
+
+// ---- fused round ------------------------------------------------------------------------
+
+bool fused_layout_ok(const brace_ctx* ctx, const float* U, int64_t ld, const void* out, int64_t out_ld) {
+  if (ctx->p.granule % 128 != 0 || ld % 4 != 0 || !aligned16(U)) return false;
+  if (ctx->p.rule == BRACE_RULE_SUM && (out_ld % 4 != 0 || !aligned16(out))) return false;
+  return true;
+}
+
+template <int VPT>
+void fused_geometry(const brace_ctx* ctx, FusedArgs& a) {
+  const int64_t tile = 256 * 4 * VPT;
+  a.tiles_per_seg = (int)((ctx->seg_max + tile - 1) / tile);
+  if (a.tiles_per_seg < 1) a.tiles_per_seg = 1;
+  a.units = (int64_t)a.tiles_per_seg * ctx->n;
+}
+
+int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t out_ld, cudaStream_t st) {
+  FusedArgs a;
+  a.pt = ctx->pt;
+  a.U = U;
+  a.ld = ld;
+  a.mail0 = ctx->mail[0];
+  a.mail1 = ctx->mail[1];
+  a.seg_pad = ctx->seg_pad;
+  a.out = out;
+  a.out_ld = out_ld;
+  a.lam = ctx->lam_i;
+  a.zs = ctx->p.zero_sign;
+  a.mean = ctx->p.mean;
+  const bool zs = ctx->p.zero_sign != 0;
+  // variant: tile width (float4 per thread per client) x clients prefetched
+  int variant = ctx->fused_variant;
+  if (variant == 0) variant = 1;
+  auto grid_for = [&](int64_t units) -> unsigned {
+    int64_t g = units;
+    if (ctx->fused_grid > 0 && g > ctx->fused_grid) g = ctx->fused_grid;
+    const int64_t cap = (int64_t)kSmCount * 4096;
+    if (g > cap) g = cap;
+    return (unsigned)(g > 0 ? g : 1);
+  };
+#define BRACE_FUSED_SIGN(VPT, UNR)                                                              \
+  do {                                                                                          \
+    fused_geometry<VPT>(ctx, a);                                                                \
+    const unsigned g = grid_for(a.units);                                                       \
+    if (ctx->entry_bytes == 1) {                                                                \
+      if (zs) fused_sign_kernel<int8_t, VPT, UNR, true><<<g, 256, 0, st>>>(a);                  \
+      else    fused_sign_kernel<int8_t, VPT, UNR, false><<<g, 256, 0, st>>>(a);                 \
+    } else {                                                                                    \
+      if (zs) fused_sign_kernel<int16_t, VPT, UNR, true><<<g, 256, 0, st>>>(a);                 \
+      else    fused_sign_kernel<int16_t, VPT, UNR, false><<<g, 256, 0, st>>>(a);                \
+    }                                                                                           \
+  } while (0)
+#define BRACE_FUSED_SUM(VPT, UNR)                                                               \
+  do {                                                                                          \
+    fused_geometry<VPT>(ctx, a);                                                                \
+    const unsigned g = grid_for(a.units);                                                       \
+    fused_sum_kernel<VPT, UNR><<<g, 256, 0, st>>>(a);                                           \
+  } while (0)
+  if (ctx->p.rule == BRACE_RULE_SUM) {
+    switch (variant) {
+      case 2: case 4: BRACE_FUSED_SUM(2, 4); break;
+      case 3: BRACE_FUSED_SUM(1, 4); break;
+      default: BRACE_FUSED_SUM(1, 8); break;
+    }
+  } else {
+    switch (variant) {
+      case 2: BRACE_FUSED_SIGN(2, 4); break;
+      case 3: BRACE_FUSED_SIGN(1, 4); break;
+      case 4: BRACE_FUSED_SIGN(2, 8); break;
+      case 5: BRACE_FUSED_SIGN(1, 16); break;
+      default: BRACE_FUSED_SIGN(1, 8); break;
+    }
+  }
+#undef BRACE_FUSED_SIGN
+#undef BRACE_FUSED_SUM
+  return check_launch(ctx);
+}
+
+// ---- argument checks shared by the ring calls -----------------------------------------------
+
+int check_device_ctx(const brace_ctx* ctx) {
+  if (!ctx) return BRACE_ERR_INVALID_ARG;
+  if (!ctx->ws) return BRACE_ERR_WORKSPACE;
+  return BRACE_OK;
+}
+
+int check_out(const brace_ctx* ctx, const void* out, int64_t out_ld) {
+  if (!out) return BRACE_ERR_INVALID_ARG;
+  const int64_t need = ctx->p.rule == BRACE_RULE_SUM ? ctx->d : (ctx->d + 31) / 32;
+  if (out_ld < need) return BRACE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(out) & 3u) != 0) return BRACE_ERR_INVALID_ARG;
+  return BRACE_OK;
+}
+
+int check_updates(const brace_ctx* ctx, const float* U, int64_t ld) {
+  if (!U || ld < ctx->d) return BRACE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(U) & 3u) != 0) return BRACE_ERR_INVALID_ARG;
+  return BRACE_OK;
+}
+
+int run_stepwise(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t out_ld, cudaStream_t st) {
+  const int n = ctx->n;
+  for (int s = 0; s < n - 1; ++s) {
+    int rc = launch_rs_step(ctx, s, U, ld, st);
+    if (rc != BRACE_OK) return rc;
+  }
+  int rc = launch_consensus(ctx, out, out_ld, st);
+  if (rc != BRACE_OK) return rc;
+  for (int t = 0; t < n - 1; ++t) {
+    rc = launch_ag_step(ctx, t, out, out_ld, st);
+    if (rc != BRACE_OK) return rc;
+  }
+  return BRACE_OK;
+}
+
+// Resolve the Byzantine id list and make sure it is on the device (Byzantine ids
+// first, honest ids after in increasing order).  The upload is skipped when the
+// device copy is already current, so steady-state calls enqueue kernels only.
+int stage_ids(brace_ctx* ctx, const int32_t* h_byz_ids, cudaStream_t st) {
+  const int n = ctx->n, f = ctx->f;
+  std::vector<int>& ids = ctx->ids_staging;
+  ids.assign((size_t)n, 0);
+  std::vector<char> is_byz((size_t)n, 0);
+  for (int b = 0; b < f; ++b) {
+    const int id = h_byz_ids ? h_byz_ids[b] : b;
+    if (id < 0 || id >= n || is_byz[(size_t)id]) return BRACE_ERR_INVALID_ARG;
+    is_byz[(size_t)id] = 1;
+    ids[(size_t)b] = id;
+  }
+  int pos = f;
+  for (int i = 0; i < n; ++i)
+    if (!is_byz[(size_t)i]) ids[(size_t)pos++] = i;
+  if (ids == ctx->ids_on_device) return BRACE_OK;
+  cudaError_t err = cudaMemcpyAsync(ctx->d_ids, ids.data(), (size_t)n * sizeof(int), cudaMemcpyHostToDevice, st);
+  if (err != cudaSuccess) return cuda_fail(ctx, err);
+  ctx->ids_on_device = ids;
+  return BRACE_OK;
+}
+
+int inject_impl(brace_ctx* ctx, const brace_attack* atk, const float* H, int64_t ld_h, float* Uo, int64_t ld_u,
+                cudaStream_t st) {
+  if (!atk) return BRACE_ERR_INVALID_ARG;
+  if (atk->kind == BRACE_ATTACK_NONE || ctx->f == 0) return BRACE_OK;
+  if (atk->kind < BRACE_ATTACK_SCALE_OWN || atk->kind > BRACE_ATTACK_SPARSE_NOISE) return BRACE_ERR_INVALID_ARG;
+  if (!H || !Uo || ld_h < ctx->d || ld_u < ctx->d) return BRACE_ERR_INVALID_ARG;
+  const int kind = atk->kind;
+  const bool needs_noise = kind == BRACE_ATTACK_GAUSSIAN || kind == BRACE_ATTACK_SPARSE_NOISE;
+  if (needs_noise && (!atk->noise || atk->noise_ld < ctx->d)) return BRACE_ERR_INVALID_ARG;
+  if (kind == BRACE_ATTACK_SPARSE_NOISE && (!atk->uniform || atk->uniform_ld < ctx->d)) return BRACE_ERR_INVALID_ARG;
+  int rc = stage_ids(ctx, atk->h_byz_ids, st);
+  if (rc != BRACE_OK) return rc;
+  if (kind == BRACE_ATTACK_SCALED_MEAN || kind == BRACE_ATTACK_MEAN_SHIFT) {
+    // two passes over the honest rows: keep the set of coordinates in flight small
+    // enough that the second pass finds the first one's lines in L2
+    int64_t blocks = (ctx->d + kThreads - 1) / kThreads;
+    const int64_t cap = (int64_t)kSmCount * 4;
+    if (blocks > cap) blocks = cap;
+    inject_stats_kernel<8><<<(unsigned)blocks, kThreads, 0, st>>>(kind, ctx->d_ids, ctx->f, ctx->n, H, ld_h, Uo, ld_u,
+                                                                 ctx->d, atk->scale, atk->kappa);
+  } else {
+    dim3 grid(tiles(ctx->d, kThreads), (unsigned)ctx->f);
+    inject_elementwise_kernel<<<grid, kThreads, 0, st>>>(kind, ctx->d_ids, H, ld_h, Uo, ld_u, atk->noise,
+                                                        atk->noise_ld, atk->uniform, atk->uniform_ld, ctx->d,
+                                                        atk->scale, atk->sigma, atk->prob);
+  }
+  return check_launch(ctx);
+}
+
+int aggregate_impl(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t out_ld, cudaStream_t st) {
+  int rc = check_updates(ctx, U, ld);
+  if (rc != BRACE_OK) return rc;
+  rc = check_out(ctx, out, out_ld);
+  if (rc != BRACE_OK) return rc;
+  const bool can_fuse = fused_layout_ok(ctx, U, ld, out, out_ld);
+  int mode = ctx->p.agg_mode;
+  if (mode == BRACE_AGG_FUSED && !can_fuse) return BRACE_ERR_UNSUPPORTED;
+  if (mode == BRACE_AGG_AUTO) mode = can_fuse ? BRACE_AGG_FUSED : BRACE_AGG_STEPWISE;
+  rc = (mode == BRACE_AGG_FUSED) ? launch_fused(ctx, U, ld, out, out_ld, st)
+                                 : run_stepwise(ctx, U, ld, out, out_ld, st);
+  if (rc != BRACE_OK) {
+    ctx->phase = kIdle;
+    return rc;
+  }
+  ctx->phase = kDone;
+  ctx->rs_done = ctx->n - 1;
+  ctx->ag_done = ctx->n - 1;
+  return BRACE_OK;
+}
+
+}  // namespace
+
+// =============================================================================================
+// C ABI
+// =============================================================================================
+extern "C" {
+
+const char* brace_status_string(int status) {
+  switch (status) {
+    case BRACE_OK: return "ok";
+    case BRACE_ERR_INVALID_ARG: return "invalid argument";
+    case BRACE_ERR_UNSUPPORTED: return "unsupported configuration";
+    case BRACE_ERR_BAD_STEP: return "ring step called out of order";
+    case BRACE_ERR_WORKSPACE: return "workspace missing, too small or misaligned";
+    case BRACE_ERR_CUDA: return "CUDA runtime error";
+    case BRACE_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int brace_default_params(brace_params* p) {
+  if (!p) return BRACE_ERR_INVALID_ARG;
+  p->rule = BRACE_RULE_SIGN_CONSENSUS;
+  p->lambda = 0.0f;
+  p->zero_sign = 0;
+  p->granule = 128;
+  p->mean = 0;
+  p->agg_mode = BRACE_AGG_AUTO;
+  return BRACE_OK;
+}
+
+size_t brace_workspace_bytes(int32_t n, int64_t d, const brace_params* params) {
+  if (n < 2 || d < 1 || !params_ok(params)) return 0;
+  return workspace_need(n, d, params);
+}
+
+int brace_init(brace_ctx** out, int32_t n, int32_t f, int64_t d, const brace_params* params, void* d_workspace,
+               size_t workspace_bytes, brace_stream_t /*stream*/) {
+  if (!out) return BRACE_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (n < 2 || f < 0 || f >= n || d < 1 || !params_ok(params)) return BRACE_ERR_INVALID_ARG;
+  const int eb = entry_bytes_for(n, params->rule);
+  if (eb == 0) return BRACE_ERR_UNSUPPORTED;
+  const size_t need = workspace_need(n, d, params);
+  const bool host_only = (d_workspace == nullptr && workspace_bytes == 0);
+  if (!host_only) {
+    if (!d_workspace || workspace_bytes < need) return BRACE_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(d_workspace) & 255u) != 0) return BRACE_ERR_WORKSPACE;
+  }
+  brace_ctx* ctx = new (std::nothrow) brace_ctx();
+  if (!ctx) return BRACE_ERR_INVALID_ARG;
+  ctx->n = n;
+  ctx->f = f;
+  ctx->d = d;
+  ctx->p = *params;
+  ctx->pt = make_part(n, d, params->granule);
+  double fl = std::floor((double)params->lambda);
+  if (fl < -(double)n - 1.0) fl = -(double)n - 1.0;
+  if (fl > (double)n) fl = (double)n;
+  ctx->lam_i = (int)fl;
+  ctx->entry_bytes = eb;
+  ctx->seg_max = longest_segment(ctx->pt);
+  ctx->seg_pad = round_up(ctx->seg_max > 0 ? ctx->seg_max : 1, kMailAlign);
+  if (!host_only) {
+    ctx->ws = static_cast<char*>(d_workspace);
+    ctx->ws_bytes = workspace_bytes;
+    const size_t one_set = (size_t)round_up((int64_t)n * ctx->seg_pad * eb, 256);
+    ctx->mail[0] = ctx->ws;
+    ctx->mail[1] = ctx->ws + one_set;
+    ctx->d_ids = reinterpret_cast<int*>(ctx->ws + 2 * one_set);
+  }
+  *out = ctx;
+  return BRACE_OK;
+}
+
+int brace_destroy(brace_ctx* ctx) {
+  if (!ctx) return BRACE_ERR_INVALID_ARG;
+  delete ctx;
+  return BRACE_OK;
+}
+
+int brace_segment(const brace_ctx* ctx, int32_t j, int64_t* begin, int64_t* end) {
+  if (!ctx || !begin || !end || j < 0 || j >= ctx->n) return BRACE_ERR_INVALID_ARG;
+  *begin = ctx->pt.begin(j);
+  *end = seg_end(ctx->pt, j);
+  return BRACE_OK;
+}
+
+int brace_last_cuda_error(const brace_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+
+int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid) {
+  if (!ctx || fused_variant < 0 || fused_variant > 5 || fused_grid < 0) return BRACE_ERR_INVALID_ARG;
+  ctx->fused_variant = fused_variant;
+  ctx->fused_grid = fused_grid;
+  return BRACE_OK;
+}
+
+int brace_inject_attack(brace_ctx* ctx, const brace_attack* attack, const float* d_honest, int64_t ld_honest,
+                        float* d_updates, int64_t ld_updates, brace_stream_t stream) {
+  int rc = check_device_ctx(ctx);
+  if (rc != BRACE_OK) return rc;
+  return inject_impl(ctx, attack, d_honest, ld_honest, d_updates, ld_updates, static_cast<cudaStream_t>(stream));
+}
+
+int brace_quantize(brace_ctx* ctx, const float* d_updates, int64_t ld, int8_t* d_q, int64_t ld_q,
+                   brace_stream_t stream) {
+  int rc = check_device_ctx(ctx);
+  if (rc != BRACE_OK) return rc;
+  rc = check_updates(ctx, d_updates, ld);
+  if (rc != BRACE_OK) return rc;
+  if (!d_q || ld_q < ctx->d) return BRACE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  dim3 grid(tiles(ctx->d, kThreads), (unsigned)ctx->n);
+  if (ctx->p.zero_sign != 0)
+    quantize_kernel<true><<<grid, kThreads, 0, st>>>(d_updates, ld, d_q, ld_q, ctx->d, ctx->p.zero_sign);
+  else
+    quantize_kernel<false><<<grid, kThreads, 0, st>>>(d_updates, ld, d_q, ld_q, ctx->d, 0);
+  return check_launch(ctx);
+}
+
+int brace_ring_reduce_scatter_step(brace_ctx* ctx, int32_t step, const float* d_updates, int64_t ld,
+                                   brace_stream_t stream) {
+  int rc = check_device_ctx(ctx);
+  if (rc != BRACE_OK) return rc;
+  rc = check_updates(ctx, d_updates, ld);
+  if (rc != BRACE_OK) return rc;
+  if (step < 0 || step > ctx->n - 2) return BRACE_ERR_BAD_STEP;
+  if (step != 0 && !(ctx->phase == kReducing && ctx->rs_done == step)) return BRACE_ERR_BAD_STEP;
+  rc = launch_rs_step(ctx, step, d_updates, ld, static_cast<cudaStream_t>(stream));
+  if (rc != BRACE_OK) {
+    ctx->phase = kIdle;
+    return rc;
+  }
+  ctx->rs_done = step + 1;
+  ctx->ag_done = 0;
+  ctx->phase = (ctx->rs_done == ctx->n - 1) ? kReduced : kReducing;
+  return BRACE_OK;
+}
+
+int brace_consensus(brace_ctx* ctx, void* d_out, int64_t out_ld, brace_stream_t stream) {
+  int rc = check_device_ctx(ctx);
+  if (rc != BRACE_OK) return rc;
+  rc = check_out(ctx, d_out, out_ld);
+  if (rc != BRACE_OK) return rc;
+  if (ctx->phase != kReduced) return BRACE_ERR_BAD_STEP;
+  rc = launch_consensus(ctx, d_out, out_ld, static_cast<cudaStream_t>(stream));
+  if (rc != BRACE_OK) {
+    ctx->phase = kIdle;
+    return rc;
+  }
+  ctx->phase = kConsensusDone;
+  ctx->ag_done = 0;
+  return BRACE_OK;
+}
+
+int brace_ring_allgather_step(brace_ctx* ctx, int32_t step, void* d_out, int64_t out_ld, brace_stream_t stream) {
+  int rc = check_device_ctx(ctx);
+  if (rc != BRACE_OK) return rc;
+  rc = check_out(ctx, d_out, out_ld);
+  if (rc != BRACE_OK) return rc;
+  if (step < 0 || step > ctx->n - 2) return BRACE_ERR_BAD_STEP;
+  const bool in_order =
+      (ctx->phase == kConsensusDone && step == 0) || (ctx->phase == kGathering && step == ctx->ag_done);
+  if (!in_order) return BRACE_ERR_BAD_STEP;
+  rc = launch_ag_step(ctx, step, d_out, out_ld, static_cast<cudaStream_t>(stream));
+  if (rc != BRACE_OK) {
+    ctx->phase = kIdle;
+    return rc;
+  }
+  ctx->ag_done = step + 1;
+  ctx->phase = (ctx->ag_done == ctx->n - 1) ? kDone : kGathering;
+  return BRACE_OK;
+}
+
+int brace_aggregate(brace_ctx* ctx, const float* d_updates, int64_t ld, void* d_out, int64_t out_ld,
+                    brace_stream_t stream) {
+  int rc = check_device_ctx(ctx);
+  if (rc != BRACE_OK) return rc;
+  return aggregate_impl(ctx, d_updates, ld, d_out, out_ld, static_cast<cudaStream_t>(stream));
+}
+
+int brace_aggregate_host(brace_ctx* ctx, const brace_attack* attack, const float* h_updates, int64_t ld, void* h_out,
+                         int64_t out_ld, float* d_updates_stage, float* d_noise_stage, float* d_uniform_stage,
+                         void* d_out_stage, brace_stream_t stream) {
+  int rc = check_device_ctx(ctx);
+  if (rc != BRACE_OK) return rc;
+  if (!h_updates || !h_out || !d_updates_stage || !d_out_stage || ld < ctx->d) return BRACE_ERR_INVALID_ARG;
+  rc = check_out(ctx, d_out_stage, out_ld);
+  if (rc != BRACE_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n = ctx->n, f = ctx->f;
+  brace_attack dev_attack;
+  const bool do_attack = attack && attack->kind != BRACE_ATTACK_NONE && f > 0;
+  if (do_attack) {
+    dev_attack = *attack;
+    const bool needs_noise = attack->kind == BRACE_ATTACK_GAUSSIAN || attack->kind == BRACE_ATTACK_SPARSE_NOISE;
+    const bool needs_unif = attack->kind == BRACE_ATTACK_SPARSE_NOISE;
+    if (needs_noise && (!attack->noise || !d_noise_stage || attack->noise_ld < ctx->d)) return BRACE_ERR_INVALID_ARG;
+    if (needs_unif && (!attack->uniform || !d_uniform_stage || attack->uniform_ld < ctx->d))
+      return BRACE_ERR_INVALID_ARG;
+    if (needs_noise) {
+      cudaError_t err = cudaMemcpyAsync(d_noise_stage, attack->noise, (size_t)f * attack->noise_ld * sizeof(float),
+                                        cudaMemcpyHostToDevice, st);
+      if (err != cudaSuccess) return cuda_fail(ctx, err);
+      dev_attack.noise = d_noise_stage;
+    }
+    if (needs_unif) {
+      cudaError_t err = cudaMemcpyAsync(d_uniform_stage, attack->uniform,
+                                        (size_t)f * attack->uniform_ld * sizeof(float), cudaMemcpyHostToDevice, st);
+      if (err != cudaSuccess) return cuda_fail(ctx, err);
+      dev_attack.uniform = d_uniform_stage;
+    }
+  }
+  cudaError_t err = cudaMemcpyAsync(d_updates_stage, h_updates, (size_t)n * ld * sizeof(float),
+                                    cudaMemcpyHostToDevice, st);
+  if (err != cudaSuccess) return cuda_fail(ctx, err);
+  if (do_attack) {
+    rc = inject_impl(ctx, &dev_attack, d_updates_stage, ld, d_updates_stage, ld, st);
+    if (rc != BRACE_OK) return rc;
+  }
+  rc = aggregate_impl(ctx, d_updates_stage, ld, d_out_stage, out_ld, st);
+  if (rc != BRACE_OK) return rc;
+  err = cudaMemcpyAsync(h_out, d_out_stage, (size_t)n * out_ld * 4, cudaMemcpyDeviceToHost, st);
+  if (err != cudaSuccess) return cuda_fail(ctx, err);
+  return BRACE_OK;
+}
+
+int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back, const void** d_ptr, int64_t* len,
+                        int32_t* segment, int32_t* entry_bytes) {
+  if (!ctx || !d_ptr || !len || client < 0 || client >= ctx->n || hops_back < 0 || hops_back > 1)
+    return BRACE_ERR_INVALID_ARG;
+  if (!ctx->ws) return BRACE_ERR_WORKSPACE;
+  if (ctx->rs_done < 1 + hops_back) return BRACE_ERR_BAD_STEP;
+  const int s = ctx->rs_done - 1 - hops_back;  // the hop asked for
+  const int set = (s + 1) & 1;
+  int j = (client - 1 - s) % ctx->n;
+  if (j < 0) j += ctx->n;
+  *d_ptr = ctx->mail[set] + (size_t)client * ctx->seg_pad * ctx->entry_bytes;
+  *len = seg_end(ctx->pt, j) - ctx->pt.begin(j);
+  if (segment) *segment = j;
+  if (entry_bytes) *entry_bytes = ctx->entry_bytes;
+  return BRACE_OK;
+}
+
+}  // extern "C"

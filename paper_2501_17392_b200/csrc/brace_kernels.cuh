@@ -1,0 +1,564 @@
+// Device kernels of the BRACE ring-aggregation library (sm_100a).
+//
+// Every kernel here is bound by HBM bandwidth (about three integer operations
+// per 4-byte element), so the design rules are: 128-bit coalesced accesses,
+// many independent loads in flight per thread, streaming cache hints for data
+// that is read once, and no re-reads of anything that can stay in registers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace brace {
+
+// ---------------------------------------------------------------------------
+// Partition of the d coordinates into n sub-vectors (Section 2.2).
+// ---------------------------------------------------------------------------
+struct Part {
+  int64_t d;   // coordinates
+  int64_t G;   // granule
+  int64_t Q;   // ceil(d / G)
+  int n;       // clients == sub-vectors
+  __host__ __device__ __forceinline__ int64_t begin(int j) const {
+    int64_t b = G * (((int64_t)j * Q) / n);
+    return b < d ? b : d;
+  }
+};
+
+__device__ __forceinline__ int next_client(int c, int n) { return c + 1 == n ? 0 : c + 1; }
+
+// Section 3 Phase I: element-wise sign.  NaN compares false both ways -> 0.
+template <bool ZS>
+__device__ __forceinline__ int sgn1(float x, int zs) {
+  int s = (int)(x > 0.0f) - (int)(x < 0.0f);
+  if (ZS) s = (x == 0.0f) ? zs : s;
+  return s;
+}
+
+// streaming (read-once) 128-bit load
+__device__ __forceinline__ float4 ld_stream(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+
+__device__ __forceinline__ void store4(int8_t* p, int a, int b, int c, int d) {
+  *reinterpret_cast<char4*>(p) = make_char4((signed char)a, (signed char)b, (signed char)c, (signed char)d);
+}
+__device__ __forceinline__ void store4(int16_t* p, int a, int b, int c, int d) {
+  *reinterpret_cast<short4*>(p) = make_short4((short)a, (short)b, (short)c, (short)d);
+}
+__device__ __forceinline__ void load4(const int8_t* p, int& a, int& b, int& c, int& d) {
+  char4 v = *reinterpret_cast<const char4*>(p);
+  a = v.x; b = v.y; c = v.z; d = v.w;
+}
+__device__ __forceinline__ void load4(const int16_t* p, int& a, int& b, int& c, int& d) {
+  short4 v = *reinterpret_cast<const short4*>(p);
+  a = v.x; b = v.y; c = v.z; d = v.w;
+}
+
+// ---------------------------------------------------------------------------
+// Share-Reduce hop, sign rule (Section 3 Phase II; Phase I fused into the read).
+// grid = (tiles over the longest sub-vector, n senders); one float4 per thread.
+// ---------------------------------------------------------------------------
+template <typename P, bool VEC, bool ZS>
+__global__ void __launch_bounds__(256)
+rs_step_sign_kernel(Part pt, const float* __restrict__ U, int64_t ld, const P* __restrict__ mail_in,
+                    P* __restrict__ mail_out, int64_t seg_pad, int step, int zs) {
+  const int n = pt.n;
+  const int c = blockIdx.y;
+  const int r = next_client(c, n);
+  int j = c - step;
+  if (j < 0) j += n;
+  const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+  const int64_t L = e - b;
+  const float* uc = U + (int64_t)c * ld + b;
+  const float* ur = U + (int64_t)r * ld + b;
+  const P* in = mail_in + (int64_t)c * seg_pad;
+  P* out = mail_out + (int64_t)r * seg_pad;
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (VEC) {
+    const int64_t i = t * 4;
+    if (i + 4 <= L) {
+      float4 x = ld_stream(ur + i);
+      int a0, a1, a2, a3;
+      if (step == 0) {
+        float4 y = ld_stream(uc + i);
+        a0 = sgn1<ZS>(y.x, zs); a1 = sgn1<ZS>(y.y, zs); a2 = sgn1<ZS>(y.z, zs); a3 = sgn1<ZS>(y.w, zs);
+      } else {
+        load4(in + i, a0, a1, a2, a3);
+      }
+      store4(out + i, a0 + sgn1<ZS>(x.x, zs), a1 + sgn1<ZS>(x.y, zs), a2 + sgn1<ZS>(x.z, zs),
+             a3 + sgn1<ZS>(x.w, zs));
+    } else {
+      for (int64_t k = i; k < L; ++k) {
+        int a = (step == 0) ? sgn1<ZS>(uc[k], zs) : (int)in[k];
+        out[k] = (P)(a + sgn1<ZS>(ur[k], zs));
+      }
+    }
+  } else {
+    if (t < L) {
+      int a = (step == 0) ? sgn1<ZS>(uc[t], zs) : (int)in[t];
+      out[t] = (P)(a + sgn1<ZS>(ur[t], zs));
+    }
+  }
+}
+
+// Share-Reduce hop, plain sum (Section 2.2 Phase I): float32 adds in ring order.
+template <bool VEC>
+__global__ void __launch_bounds__(256)
+rs_step_sum_kernel(Part pt, const float* __restrict__ U, int64_t ld, const float* __restrict__ mail_in,
+                   float* __restrict__ mail_out, int64_t seg_pad, int step) {
+  const int n = pt.n;
+  const int c = blockIdx.y;
+  const int r = next_client(c, n);
+  int j = c - step;
+  if (j < 0) j += n;
+  const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+  const int64_t L = e - b;
+  const float* uc = U + (int64_t)c * ld + b;
+  const float* ur = U + (int64_t)r * ld + b;
+  const float* in = (step == 0) ? uc : mail_in + (int64_t)c * seg_pad;
+  float* out = mail_out + (int64_t)r * seg_pad;
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (VEC) {
+    const int64_t i = t * 4;
+    if (i + 4 <= L) {
+      float4 x = ld_stream(ur + i);
+      float4 y = (step == 0) ? ld_stream(in + i) : *reinterpret_cast<const float4*>(in + i);
+      float4 o;
+      o.x = __fadd_rn(y.x, x.x); o.y = __fadd_rn(y.y, x.y); o.z = __fadd_rn(y.z, x.z); o.w = __fadd_rn(y.w, x.w);
+      *reinterpret_cast<float4*>(out + i) = o;
+    } else {
+      for (int64_t k = i; k < L; ++k) out[k] = __fadd_rn(in[k], ur[k]);
+    }
+  } else {
+    if (t < L) out[t] = __fadd_rn(in[t], ur[t]);
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Consensus, Eq. (1): one thread per 32-bit output word of the owner's sub-vector.
+// Words that straddle a sub-vector boundary (granule % 32 != 0) are
+// read-modify-written; in one launch each row is written by one sub-vector only.
+// ---------------------------------------------------------------------------
+template <typename P>
+__global__ void __launch_bounds__(256)
+consensus_sign_kernel(Part pt, const P* __restrict__ mail, int64_t seg_pad, uint32_t* __restrict__ out,
+                      int64_t out_ld, int lam) {
+  const int n = pt.n;
+  const int c = blockIdx.y;
+  const int j = next_client(c, n);
+  const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+  if (b >= e) return;
+  const int64_t w0 = b >> 5, w1 = (e + 31) >> 5;
+  const int64_t w = w0 + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (w >= w1) return;
+  const int64_t k0 = (w << 5) > b ? (w << 5) : b;
+  const int64_t k1 = ((w + 1) << 5) < e ? ((w + 1) << 5) : e;
+  const P* src = mail + (int64_t)c * seg_pad;      // src[k - b] is coordinate k
+  uint32_t bits = 0;
+  if (k1 - k0 == 32 && ((k0 - b) & 15) == 0) {
+    constexpr int NV = (int)(32 * sizeof(P) / 16);
+    uint4 raw[NV];
+#pragma unroll
+    for (int q = 0; q < NV; ++q) raw[q] = reinterpret_cast<const uint4*>(src + (k0 - b))[q];
+    const P* v = reinterpret_cast<const P*>(raw);
+#pragma unroll
+    for (int q = 0; q < 32; ++q) bits |= (uint32_t)((int)v[q] > lam) << q;
+  } else {
+    for (int64_t k = k0; k < k1; ++k) bits |= (uint32_t)((int)src[k - b] > lam) << (int)(k & 31);
+  }
+  const int lo = (int)(k0 & 31);
+  int hi = (int)(k1 - (w << 5));                    // one past the last bit this sub-vector owns
+  if (k1 == pt.d) hi = 32;                          // bits past d are padding: written as 0
+  const uint32_t mask = (hi == 32 ? 0xffffffffu : ((1u << hi) - 1u)) & ~((1u << lo) - 1u);
+  uint32_t* dst = out + (int64_t)c * out_ld + w;
+  *dst = (mask == 0xffffffffu) ? bits : ((*dst & ~mask) | bits);
+}
+
+// Phase III under the plain-sum rule: identity, or division by n.
+template <bool VEC>
+__global__ void __launch_bounds__(256)
+consensus_sum_kernel(Part pt, const float* __restrict__ mail, int64_t seg_pad, float* __restrict__ out,
+                     int64_t out_ld, int mean) {
+  const int n = pt.n;
+  const int c = blockIdx.y;
+  const int j = next_client(c, n);
+  const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+  const int64_t L = e - b;
+  const float* src = mail + (int64_t)c * seg_pad;
+  float* dst = out + (int64_t)c * out_ld + b;
+  const float fn = (float)n;
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (VEC) {
+    const int64_t i = t * 4;
+    if (i + 4 <= L) {
+      float4 v = *reinterpret_cast<const float4*>(src + i);
+      if (mean) { v.x = __fdiv_rn(v.x, fn); v.y = __fdiv_rn(v.y, fn); v.z = __fdiv_rn(v.z, fn); v.w = __fdiv_rn(v.w, fn); }
+      *reinterpret_cast<float4*>(dst + i) = v;
+    } else {
+      for (int64_t k = i; k < L; ++k) dst[k] = mean ? __fdiv_rn(src[k], fn) : src[k];
+    }
+  } else {
+    if (t < L) dst[t] = mean ? __fdiv_rn(src[t], fn) : src[t];
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Share-Only hop (Section 3 Phase IV): row c -> row (c+1) mod n, one sub-vector.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+ag_step_bits_kernel(Part pt, uint32_t* out, int64_t out_ld, int step) {
+  const int n = pt.n;
+  const int c = blockIdx.y;
+  const int r = next_client(c, n);
+  int j = c + 1 - step;
+  if (j < 0) j += n;
+  if (j >= n) j -= n;
+  const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+  if (b >= e) return;
+  const int64_t w0 = b >> 5, w1 = (e + 31) >> 5;
+  const int64_t w = w0 + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (w >= w1) return;
+  const int64_t k0 = (w << 5) > b ? (w << 5) : b;
+  const int64_t k1 = ((w + 1) << 5) < e ? ((w + 1) << 5) : e;
+  const int lo = (int)(k0 & 31);
+  int hi = (int)(k1 - (w << 5));
+  if (k1 == pt.d) hi = 32;
+  const uint32_t mask = (hi == 32 ? 0xffffffffu : ((1u << hi) - 1u)) & ~((1u << lo) - 1u);
+  const uint32_t v = out[(int64_t)c * out_ld + w];
+  uint32_t* dst = out + (int64_t)r * out_ld + w;
+  *dst = (mask == 0xffffffffu) ? v : ((*dst & ~mask) | (v & mask));
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(256)
+ag_step_f32_kernel(Part pt, float* out, int64_t out_ld, int step) {
+  const int n = pt.n;
+  const int c = blockIdx.y;
+  const int r = next_client(c, n);
+  int j = c + 1 - step;
+  if (j < 0) j += n;
+  if (j >= n) j -= n;
+  const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+  const int64_t L = e - b;
+  const float* src = out + (int64_t)c * out_ld + b;
+  float* dst = out + (int64_t)r * out_ld + b;
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (VEC) {
+    const int64_t i = t * 4;
+    if (i + 4 <= L) {
+      *reinterpret_cast<float4*>(dst + i) = *reinterpret_cast<const float4*>(src + i);
+    } else {
+      for (int64_t k = i; k < L; ++k) dst[k] = src[k];
+    }
+  } else {
+    if (t < L) dst[t] = src[t];
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Fused round: a CTA takes one tile of one sub-vector j and walks it through the
+// ring in hop order -- client j, j+1, .., j+n-1 -- keeping the partial that
+// would travel on the wire in registers.  The loads of the next UNR clients'
+// rows are issued before the current ones are consumed (their addresses do not
+// depend on data).  Only the partials of the last two hops are stored to the
+// mailboxes: those are the only mailbox contents that survive a round in the
+// hop-by-hop execution, so the final buffer state is the same.  The tile's
+// consensus bits are staged in shared memory and written to all n output rows
+// (what Share-Only leaves behind).
+// ---------------------------------------------------------------------------
+struct FusedArgs {
+  Part pt;
+  const float* U;
+  int64_t ld;
+  void* mail0;
+  void* mail1;
+  int64_t seg_pad;
+  void* out;
+  int64_t out_ld;
+  int lam;
+  int zs;
+  int mean;
+  int tiles_per_seg;
+  int64_t units;
+};
+
+template <typename P, int VPT, int UNR, bool ZS>
+__global__ void __launch_bounds__(256)
+fused_sign_kernel(const FusedArgs a) {
+  static_assert(VPT >= 1 && VPT <= 8, "tile width");
+  constexpr int TILE = 256 * 4 * VPT;
+  constexpr int WPT = 32 * VPT;                    // output words per tile
+  __shared__ uint32_t sm_words[WPT];
+  const Part pt = a.pt;
+  const int n = pt.n;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* __restrict__ U = a.U;
+  uint32_t* __restrict__ out = reinterpret_cast<uint32_t*>(a.out);
+
+  for (int64_t u = blockIdx.x; u < a.units; u += gridDim.x) {
+    const int j = (int)(u / a.tiles_per_seg);
+    const int k = (int)(u % a.tiles_per_seg);
+    const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+    const int64_t L = e - b;
+    const int64_t t0 = (int64_t)k * TILE;
+    if (t0 >= L) continue;                         // uniform over the CTA
+
+    int64_t off[VPT];
+    int nv[VPT];
+    int acc[VPT][4];
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+      off[v] = t0 + (int64_t)(v * 256 + tid) * 4;
+      const int64_t rem = L - off[v];
+      nv[v] = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
+      acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0;
+    }
+    const float* base = U + b;
+    int c = j;
+    for (int i0 = 0; i0 < n; i0 += UNR) {
+      float4 x[UNR][VPT];
+      int cc = c;
+#pragma unroll
+      for (int q = 0; q < UNR; ++q) {
+        if (i0 + q < n) {
+          const float* row = base + (int64_t)cc * a.ld;
+#pragma unroll
+          for (int v = 0; v < VPT; ++v)
+            x[q][v] = nv[v] > 0 ? ld_stream(row + off[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
+          cc = next_client(cc, n);
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < UNR; ++q) {
+        if (i0 + q < n) {
+          const int i = i0 + q;
+#pragma unroll
+          for (int v = 0; v < VPT; ++v) {
+            acc[v][0] += sgn1<ZS>(x[q][v].x, a.zs);
+            acc[v][1] += sgn1<ZS>(x[q][v].y, a.zs);
+            acc[v][2] += sgn1<ZS>(x[q][v].z, a.zs);
+            acc[v][3] += sgn1<ZS>(x[q][v].w, a.zs);
+          }
+          if (i >= 1 && i >= n - 2) {              // hop s = i-1 lands in client c's mailbox, set (s+1)&1
+            P* m = reinterpret_cast<P*>((i & 1) ? a.mail1 : a.mail0) + (int64_t)c * a.seg_pad;
+#pragma unroll
+            for (int v = 0; v < VPT; ++v) {
+              if (nv[v] == 4) {
+                store4(m + off[v], acc[v][0], acc[v][1], acc[v][2], acc[v][3]);
+              } else {
+#pragma unroll
+                for (int q2 = 0; q2 < 3; ++q2)
+                  if (q2 < nv[v]) m[off[v] + q2] = (P)acc[v][q2];
+              }
+            }
+          }
+          c = next_client(c, n);
+        }
+      }
+    }
+
+    // consensus bits: 4 per thread, 8 lanes make one word
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+      uint32_t nib = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) nib |= (uint32_t)(q < nv[v] && acc[v][q] > a.lam) << q;
+      uint32_t word = nib << (4 * (lane & 7));
+      word |= __shfl_xor_sync(0xffffffffu, word, 1);
+      word |= __shfl_xor_sync(0xffffffffu, word, 2);
+      word |= __shfl_xor_sync(0xffffffffu, word, 4);
+      if ((lane & 7) == 0) sm_words[v * 32 + warp * 4 + (lane >> 3)] = word;
+    }
+    __syncthreads();
+    const int64_t left = L - t0;
+    const int nw = left >= TILE ? WPT : (int)((left + 31) >> 5);
+    const int64_t wb = (b + t0) >> 5;
+    const int w = tid % WPT;
+    if (w < nw) {
+      const uint32_t val = sm_words[w];
+      for (int row = tid / WPT; row < n; row += 256 / WPT) out[(int64_t)row * a.out_ld + wb + w] = val;
+    }
+    __syncthreads();
+  }
+}
+
+template <int VPT, int UNR>
+__global__ void __launch_bounds__(256)
+fused_sum_kernel(const FusedArgs a) {
+  constexpr int TILE = 256 * 4 * VPT;
+  const Part pt = a.pt;
+  const int n = pt.n;
+  const int tid = threadIdx.x;
+  const float* __restrict__ U = a.U;
+  float* __restrict__ out = reinterpret_cast<float*>(a.out);
+  const float fn = (float)n;
+
+  for (int64_t u = blockIdx.x; u < a.units; u += gridDim.x) {
+    const int j = (int)(u / a.tiles_per_seg);
+    const int k = (int)(u % a.tiles_per_seg);
+    const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+    const int64_t L = e - b;
+    const int64_t t0 = (int64_t)k * TILE;
+    if (t0 >= L) continue;
+
+    int64_t off[VPT];
+    int nv[VPT];
+    float acc[VPT][4];
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+      off[v] = t0 + (int64_t)(v * 256 + tid) * 4;
+      const int64_t rem = L - off[v];
+      nv[v] = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
+      acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0.f;
+    }
+    const float* base = U + b;
+    int c = j;
+    for (int i0 = 0; i0 < n; i0 += UNR) {
+      float4 x[UNR][VPT];
+      int cc = c;
+#pragma unroll
+      for (int q = 0; q < UNR; ++q) {
+        if (i0 + q < n) {
+          const float* row = base + (int64_t)cc * a.ld;
+#pragma unroll
+          for (int v = 0; v < VPT; ++v)
+            x[q][v] = nv[v] > 0 ? ld_stream(row + off[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
+          cc = next_client(cc, n);
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < UNR; ++q) {
+        if (i0 + q < n) {
+          const int i = i0 + q;
+#pragma unroll
+          for (int v = 0; v < VPT; ++v) {
+            if (i == 0) {                          // the sub-vector starts as client j's own values
+              acc[v][0] = x[q][v].x; acc[v][1] = x[q][v].y; acc[v][2] = x[q][v].z; acc[v][3] = x[q][v].w;
+            } else {                               // received partial + own, float32, ring order
+              acc[v][0] = __fadd_rn(acc[v][0], x[q][v].x);
+              acc[v][1] = __fadd_rn(acc[v][1], x[q][v].y);
+              acc[v][2] = __fadd_rn(acc[v][2], x[q][v].z);
+              acc[v][3] = __fadd_rn(acc[v][3], x[q][v].w);
+            }
+          }
+          if (i >= 1 && i >= n - 2) {
+            float* m = reinterpret_cast<float*>((i & 1) ? a.mail1 : a.mail0) + (int64_t)c * a.seg_pad;
+#pragma unroll
+            for (int v = 0; v < VPT; ++v) {
+              if (nv[v] == 4) {
+                *reinterpret_cast<float4*>(m + off[v]) = make_float4(acc[v][0], acc[v][1], acc[v][2], acc[v][3]);
+              } else {
+#pragma unroll
+                for (int q2 = 0; q2 < 3; ++q2)
+                  if (q2 < nv[v]) m[off[v] + q2] = acc[v][q2];
+              }
+            }
+          }
+          c = next_client(c, n);
+        }
+      }
+    }
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+      if (a.mean) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[v][q] = __fdiv_rn(acc[v][q], fn);
+      }
+      float* dst = out + b + off[v];
+      if (nv[v] == 4) {
+        const float4 val = make_float4(acc[v][0], acc[v][1], acc[v][2], acc[v][3]);
+        for (int row = 0; row < n; ++row) *reinterpret_cast<float4*>(dst + (int64_t)row * a.out_ld) = val;
+      } else {
+        for (int row = 0; row < n; ++row) {
+#pragma unroll
+          for (int q = 0; q < 3; ++q)
+            if (q < nv[v]) dst[(int64_t)row * a.out_ld + q] = acc[v][q];
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Phase I on its own (inspection / tests): int8 sign matrix.
+// ---------------------------------------------------------------------------
+template <bool ZS>
+__global__ void __launch_bounds__(256)
+quantize_kernel(const float* __restrict__ U, int64_t ld, int8_t* __restrict__ q, int64_t ld_q, int64_t d, int zs) {
+  const int c = blockIdx.y;
+  const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (k < d) q[(int64_t)c * ld_q + k] = (int8_t)sgn1<ZS>(U[(int64_t)c * ld + k], zs);
+}
+
+// ---------------------------------------------------------------------------
+// Byzantine alterations (threat model of Section 3), applied before the ring.
+// ids[0..f) are the Byzantine clients, ids[f..n) the honest ones in increasing id.
+// ---------------------------------------------------------------------------
+// kinds 1, 2, 5: element-wise, grid = (tiles over d, f Byzantine rows)
+__global__ void __launch_bounds__(256)
+inject_elementwise_kernel(int kind, const int* __restrict__ ids, const float* H, int64_t ld_h,
+                          float* Uo, int64_t ld_u, const float* __restrict__ noise, int64_t ld_z,
+                          const float* __restrict__ unif, int64_t ld_r, int64_t d, float scale, float sigma,
+                          float prob) {
+  const int bidx = blockIdx.y;
+  const int id = ids[bidx];
+  const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= d) return;
+  float v;
+  if (kind == 1) {
+    v = __fmul_rn(scale, H[(int64_t)id * ld_h + k]);
+  } else if (kind == 2) {
+    v = __fmul_rn(sigma, noise[(int64_t)bidx * ld_z + k]);
+  } else {
+    const float z = __fmul_rn(sigma, noise[(int64_t)bidx * ld_z + k]);
+    v = (unif[(int64_t)bidx * ld_r + k] < prob) ? z : 0.0f;
+  }
+  Uo[(int64_t)id * ld_u + k] = v;
+}
+
+// kinds 3, 4: per-coordinate mean (and population std, two passes) over the
+// honest rows in float64, rounded once to float32, written to every Byzantine row.
+// No fused multiply-add anywhere: each operation rounds on its own.
+template <int UNR>
+__global__ void __launch_bounds__(256)
+inject_stats_kernel(int kind, const int* __restrict__ ids, int f, int n, const float* H, int64_t ld_h,
+                    float* Uo, int64_t ld_u, int64_t d, float scale, float kappa) {
+  const int m = n - f;
+  const int* good = ids + f;
+  for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < d; k += (int64_t)gridDim.x * blockDim.x) {
+    double total = 0.0;
+    for (int i0 = 0; i0 < m; i0 += UNR) {
+      float x[UNR];
+#pragma unroll
+      for (int q = 0; q < UNR; ++q)
+        if (i0 + q < m) x[q] = H[(int64_t)good[i0 + q] * ld_h + k];
+#pragma unroll
+      for (int q = 0; q < UNR; ++q)
+        if (i0 + q < m) total = __dadd_rn(total, (double)x[q]);
+    }
+    const double mean = __ddiv_rn(total, (double)m);
+    double vec;
+    if (kind == 3) {
+      vec = __dmul_rn((double)scale, mean);
+    } else {
+      double sq = 0.0;
+      for (int i0 = 0; i0 < m; i0 += UNR) {
+        float x[UNR];
+#pragma unroll
+        for (int q = 0; q < UNR; ++q)
+          if (i0 + q < m) x[q] = H[(int64_t)good[i0 + q] * ld_h + k];
+#pragma unroll
+        for (int q = 0; q < UNR; ++q)
+          if (i0 + q < m) {
+            const double dev = __dsub_rn((double)x[q], mean);
+            sq = __dadd_rn(sq, __dmul_rn(dev, dev));
+          }
+      }
+      const double sd = __dsqrt_rn(__ddiv_rn(sq, (double)m));
+      vec = __dsub_rn(mean, __dmul_rn((double)kappa, sd));
+    }
+    const float v = __double2float_rn(vec);
+    for (int bq = 0; bq < f; ++bq) Uo[(int64_t)ids[bq] * ld_u + k] = v;
+  }
+}
+
+}  // namespace brace
