@@ -1,0 +1,434 @@
+"""Parity of the CUDA library against the CPU oracle, through the C ABI.
+
+Integer work (signs, per-hop partial sign-sums, consensus bits, every client's
+output row) must match bit for bit.  The plain-sum rule must match the oracle's
+float32 ring-order sum bit for bit and the float64 sum within 1e-5 relative to
+sum_i |g_i[k]| (the textbook forward-error scale of an n-term float32 sum)."""
+
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import brace_oracle as O
+from paper_2501_17392_b200 import brace as B
+from paper_2501_17392_b200 import build as brace_build
+from paper_2501_17392_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+REL_TOL = 1e-5
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    brace_build.build()
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+
+
+def dev(x: np.ndarray | torch.Tensor) -> torch.Tensor:
+    t = torch.as_tensor(x)
+    return t.cuda()
+
+
+def expected_words(pm1_row: np.ndarray, d: int) -> np.ndarray:
+    return O.pack_bits_fast(pm1_row, words=(d + 31) // 32)
+
+
+def out_words(out: torch.Tensor, d: int) -> np.ndarray:
+    """[n, ceil(d/32)] uint32 view of the library's output rows."""
+    return out[:, : (d + 31) // 32].cpu().numpy().view(np.uint32)
+
+
+def run_steps_and_check(ctx: B.Brace, U: torch.Tensor, tr: O.RingTrace, out: torch.Tensor, rule: int, d: int):
+    """Drive the ring hop by hop; compare every client's mailbox after every hop."""
+    n = ctx.n
+    for s in range(n - 1):
+        ctx.reduce_scatter_step(s, U)
+        for r in range(n):
+            seg, got = ctx.mailbox_tensor(r)
+            exp_seg, exp = tr.rs_states[s][r]
+            assert seg == exp_seg, (s, r)
+            if rule == B.RULE_SUM:
+                assert np.array_equal(got.numpy().view(np.uint32), exp.view(np.uint32)), (s, r)
+            else:
+                assert np.array_equal(got.numpy().astype(np.int32), exp), (s, r)
+    ctx.consensus(out)
+    for t in range(n - 1):
+        ctx.allgather_step(t, out)
+        if rule != B.RULE_SUM and tr.ag_states:
+            # after hop t client r holds sub-vectors r+1, r, .., r-t (mod n) -- check the newest
+            got = out_words(out, d)
+            for r in range(n):
+                j = (r - t) % n
+                b, e = tr.bounds[j]
+                bits = np.unpackbits(got[r].view(np.uint8), bitorder="little")[b:e]
+                assert np.array_equal(bits, (tr.ag_states[t][r][b:e] > 0).astype(np.uint8)), (t, r)
+
+
+def check_final(out: torch.Tensor, tr: O.RingTrace, rule: int, d: int):
+    n = tr.outputs.shape[0]
+    if rule == B.RULE_SUM:
+        got = out[:, :d].cpu().numpy()
+        for c in range(n):
+            assert np.array_equal(got[c].view(np.uint32), tr.outputs[c].view(np.uint32)), c
+    else:
+        got = out_words(out, d)
+        exp = expected_words(tr.outputs[0], d)
+        for c in range(n):
+            assert np.array_equal(got[c], exp), c
+
+
+def final_mailboxes(ctx: B.Brace):
+    return [[ctx.mailbox_tensor(c, hb) for c in range(ctx.n)] for hb in range(2 if ctx.n > 2 else 1)]
+
+
+# ------------------------------------------------------------------ brute force on tiny inputs
+@pytest.mark.parametrize("n", [2, 3, 4, 5])
+def test_brute_force_all_sign_patterns(n):
+    """All 3^n sign patterns at every coordinate, d = 1..8, lambda sweep, granules 1 / 2 / 128."""
+    patterns = list(itertools.product([0, 1, 2], repeat=n))
+    P = len(patterns)
+    mags = np.array([0.5, 3.0, 1e-30, 7e20], dtype=np.float32)
+    for d in range(1, 9):
+        ld = 8
+        out = torch.zeros((n, 4), dtype=torch.int32, device="cuda")
+        for m in range(P):
+            U = np.zeros((n, ld), dtype=np.float32)
+            pats = [patterns[(m + k) % P] for k in range(d)]
+            for k, pat in enumerate(pats):
+                for i, t in enumerate(pat):
+                    U[i, k] = (t - 1) * mags[(i + k) % 4]
+            Ud = dev(U)
+            settings = [(lam, 1) for lam in range(-n - 1, n + 1)] + [(lam, G) for G in (2, 128) for lam in (-1, 0, 1)]
+            if m % 9:
+                settings = [(0, 1), (1, 2), (-1, 128)]
+            for lam, G in settings:
+                tr = O.ring_round(U[:, :d], lam=lam, granule=G, keep_states=(m % 27 == 0))
+                ctx = B.Brace(n, 0, d, B.default_params(lam=float(lam), granule=G))
+                out.fill_(-1)
+                if m % 27 == 0:
+                    run_steps_and_check(ctx, Ud, tr, out, B.RULE_SIGN_CONSENSUS, d)
+                    check_final(out, tr, B.RULE_SIGN_CONSENSUS, d)
+                    out.fill_(-1)
+                ctx.aggregate(Ud, out)
+                check_final(out, tr, B.RULE_SIGN_CONSENSUS, d)
+                ctx.close()
+
+
+# ------------------------------------------------------------------ medium cases: several tiles + ragged tails
+CASES = [
+    # n, d, G, ld, lam, zero_sign
+    (8, 100_000, 128, 100_096, 0.0, 0),
+    (20, 70_001, 128, 70_004, 1.0, 0),
+    (5, 4_099, 128, 4_100, 0.5, 1),
+    (3, 1_000, 32, 1_000, 2.0, 0),
+    (7, 12_345, 4, 12_348, -1.0, -1),
+    (13, 50_001, 1, 50_001, 0.0, 0),
+    (6, 33_000, 128, 33_024, 1.0, 0),
+    (2, 5_000, 128, 5_000, 0.0, 0),
+    (16, 300, 128, 384, 0.0, 0),          # fewer granules than clients: empty sub-vectors
+    (9, 2_049, 128, 2_052, 3.0, 0),
+]
+
+
+@pytest.mark.parametrize("n,d,G,ld,lam,zs", CASES)
+@pytest.mark.parametrize("rule", [B.RULE_SIGN_CONSENSUS, B.RULE_SUM])
+def test_hop_by_hop_and_whole_round(n, d, G, ld, lam, zs, rule):
+    U = W.small_integer_updates(n, d, seed=n + d, ld=ld) if (d % 2) else None
+    if U is None:
+        g = torch.Generator().manual_seed(n * 7 + d)
+        U = torch.zeros((n, ld), dtype=torch.float32)
+        U[:, :d].normal_(generator=g)
+        U[:, :d][torch.rand((n, d), generator=g) < 0.15] = 0.0
+    U[:, d:] = 123.0                                    # padding must never be read as data
+    Uh = U.numpy()[:, :d]
+    mean = 1 if (rule == B.RULE_SUM and n % 2) else 0
+    tr = O.ring_round(Uh, rule=rule, lam=lam, zero_sign=zs, granule=G, mean=bool(mean))
+    Ud = U.cuda()
+    fusable = (G % 128 == 0) and (ld % 4 == 0)
+
+    # (1) step calls, with per-hop parity
+    ctx = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, zero_sign=zs, granule=G, mean=mean,
+                                            agg_mode=B.AGG_STEPWISE))
+    out = ctx.new_output()
+    out.fill_(-7 if rule != B.RULE_SUM else 0)
+    run_steps_and_check(ctx, Ud, tr, out, rule, d)
+    check_final(out, tr, rule, d)
+    if rule == B.RULE_SIGN_CONSENSUS:
+        assert np.array_equal(O.gar_direct(Uh, lam, zs), tr.outputs[0])
+    boxes_steps = final_mailboxes(ctx)
+
+    # (2) whole round, stepwise launches
+    out2 = torch.full_like(out, 5)
+    ctx.aggregate(Ud, out2)
+    check_final(out2, tr, rule, d)
+
+    # (3) whole round, fused kernel, every shape; mailboxes end as the step calls left them
+    if fusable:
+        for variant in range(0, 6):
+            ctxf = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, zero_sign=zs, granule=G, mean=mean,
+                                                     agg_mode=B.AGG_FUSED))
+            ctxf.workspace.fill_(0x5A)
+            ctxf.set_tuning(variant, 3 if variant == 2 else 0)
+            out3 = torch.full_like(out, 9)
+            ctxf.aggregate(Ud, out3)
+            check_final(out3, tr, rule, d)
+            boxes_fused = final_mailboxes(ctxf)
+            for hb in range(len(boxes_steps)):
+                for c in range(n):
+                    seg_a, a = boxes_steps[hb][c]
+                    seg_b, b2 = boxes_fused[hb][c]
+                    assert seg_a == seg_b
+                    assert torch.equal(a.view(torch.uint8), b2.view(torch.uint8)), (variant, hb, c)
+            ctxf.close()
+    else:
+        ctxf = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, zero_sign=zs, granule=G, agg_mode=B.AGG_FUSED))
+        assert ctxf.aggregate_status(Ud, torch.zeros_like(out)) == B.ERR_UNSUPPORTED
+        ctxf.close()
+        ctxa = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, zero_sign=zs, granule=G, mean=mean))
+        out4 = torch.full_like(out, 3)
+        ctxa.aggregate(Ud, out4)                        # AUTO falls back to stepwise launches
+        check_final(out4, tr, rule, d)
+        ctxa.close()
+
+    # (4) plain sum against float64, relative to sum |g_i|
+    if rule == B.RULE_SUM:
+        ref = O.sum_direct_f64(Uh) / (n if mean else 1)
+        scale = np.sum(np.abs(Uh.astype(np.float64)), axis=0) / (n if mean else 1)
+        got = out2[0, :d].cpu().numpy().astype(np.float64)
+        assert (np.abs(got - ref) <= REL_TOL * np.maximum(np.abs(ref), scale) + 1e-30).all()
+    ctx.close()
+
+
+def test_unaligned_rows_fall_back_to_scalar_kernels():
+    """Row stride not a multiple of 4 and a base pointer off 16 bytes."""
+    n, d, ld = 6, 3_001, 3_003
+    g = torch.Generator().manual_seed(5)
+    buf = torch.zeros(n * ld + 1, dtype=torch.float32)
+    buf.normal_(generator=g)
+    Ud_full = buf.cuda()
+    Ud = Ud_full[1:].view(n, ld)                        # 4-byte aligned only
+    Uh = buf[1:].view(n, ld)[:, :d].numpy()
+    for rule in (B.RULE_SIGN_CONSENSUS, B.RULE_SUM):
+        tr = O.ring_round(Uh, rule=rule, lam=1.0, granule=128)
+        ctx = B.Brace(n, 0, d, B.default_params(rule=rule, lam=1.0))
+        out = ctx.new_output(out_ld=(d + 1) if rule == B.RULE_SUM else None)
+        run_steps_and_check(ctx, Ud, tr, out, rule, d)
+        check_final(out, tr, rule, d)
+        out.zero_()
+        ctx.aggregate(Ud, out)
+        check_final(out, tr, rule, d)
+        ctx.close()
+
+
+def test_special_float_values():
+    n, d = 9, 10_000
+    U = W.edge_value_updates(n, d, seed=3, ld=10_112)
+    Uh = U.numpy()[:, :d]
+    for zs in (0, 1, -1):
+        for lam in (0.0, -2.0, 2.5):
+            tr = O.ring_round(Uh, lam=lam, zero_sign=zs, keep_states=False)
+            ctx = B.Brace(n, 0, d, B.default_params(lam=lam, zero_sign=zs))
+            out = ctx.new_output()
+            ctx.aggregate(U.cuda(), out)
+            check_final(out, tr, B.RULE_SIGN_CONSENSUS, d)
+            ctx.close()
+    # Phase I on its own
+    ctx = B.Brace(n, 0, d)
+    q = torch.zeros((n, d), dtype=torch.int8, device="cuda")
+    ctx.quantize(U.cuda(), q)
+    assert np.array_equal(q.cpu().numpy().astype(np.int32), O.sgn(Uh))
+    ctx.close()
+
+
+@pytest.mark.parametrize("n", [127, 128, 300])
+def test_many_clients_partial_width(n):
+    """int8 partial sums up to n = 127, int16 beyond; unanimous columns reach +-n."""
+    d = 20_000
+    g = torch.Generator().manual_seed(n)
+    U = torch.zeros((n, d), dtype=torch.float32)
+    U.normal_(generator=g)
+    U[:, :64] = 1.0
+    U[:, 64:128] = -1.0
+    Uh = U.numpy()
+    lam = float(n - 1)
+    tr = O.ring_round(Uh, lam=lam, keep_states=False)
+    assert tr.outputs[0][:64].tolist() == [1] * 64
+    for mode in (B.AGG_STEPWISE, B.AGG_FUSED):
+        ctx = B.Brace(n, 0, d, B.default_params(lam=lam, agg_mode=mode))
+        out = ctx.new_output()
+        ctx.aggregate(U.cuda(), out)
+        check_final(out, tr, B.RULE_SIGN_CONSENSUS, d)
+        j, owned = ctx.mailbox_tensor(n - 1)             # client n-1 owns sub-vector 0
+        assert j == 0
+        assert np.array_equal(owned.numpy().astype(np.int32), tr.owned[n - 1][1])
+        ctx.close()
+
+
+def test_rounds_are_memoryless():
+    """Five consecutive rounds on one context equal five rounds on fresh contexts."""
+    w = W.scaled(W.WORKLOADS["cfg5"], 40_000)
+    ctx = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam))
+    out = ctx.new_output()
+    for rnd in range(5):
+        U = W.honest_updates(w, rnd, device="cuda")
+        ctx.aggregate(U, out)
+        fresh = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam, agg_mode=B.AGG_STEPWISE))
+        out_f = fresh.new_output()
+        fresh.aggregate(U, out_f)
+        assert torch.equal(out, out_f)
+        tr = O.ring_round(U.cpu().numpy()[:, :w.d], lam=w.lam, keep_states=False)
+        check_final(out, tr, B.RULE_SIGN_CONSENSUS, w.d)
+        fresh.close()
+    ctx.close()
+
+
+def test_guard_bands_stay_untouched():
+    """Canaries around the workspace, the output and the mailbox tails."""
+    n, d, ld = 7, 9_001, 9_004
+    g = torch.Generator().manual_seed(1)
+    U = torch.zeros((n, ld), dtype=torch.float32)
+    U[:, :d].normal_(generator=g)
+    Ud = U.cuda()
+    for rule in (B.RULE_SIGN_CONSENSUS, B.RULE_SUM):
+        for mode in (B.AGG_STEPWISE, B.AGG_FUSED):
+            p = B.default_params(rule=rule, agg_mode=mode)
+            need = B.workspace_bytes(n, d, p)
+            guard = 4096
+            raw = torch.full((need + 2 * guard,), 0xA5, dtype=torch.uint8, device="cuda")
+            ctx = B.Brace(n, 0, d, p, workspace=raw[guard: guard + need])
+            words = (d + 31) // 32
+            out_ld = (d + 4) if rule == B.RULE_SUM else words + 3
+            if rule == B.RULE_SUM:
+                out_ld = (out_ld + 3) // 4 * 4
+            outbuf = torch.full((n + 2, out_ld), 0x3C3C3C3C, dtype=torch.int32, device="cuda")
+            out = outbuf[1: n + 1]
+            if rule == B.RULE_SUM:
+                out = out.view(torch.float32)
+            ctx.aggregate(Ud, out)
+            torch.cuda.synchronize()
+            assert (raw[:guard] == 0xA5).all() and (raw[guard + need:] == 0xA5).all()
+            assert (outbuf[0] == 0x3C3C3C3C).all() and (outbuf[n + 1] == 0x3C3C3C3C).all()
+            used = d if rule == B.RULE_SUM else words
+            assert (outbuf[1: n + 1, used:] == 0x3C3C3C3C).all()
+            tr = O.ring_round(U.numpy()[:, :d], rule=rule, keep_states=False)
+            check_final(out, tr, rule, d)
+            ctx.close()
+
+
+# ------------------------------------------------------------------ API errors: status code, nothing launched
+def test_step_order_and_argument_errors():
+    n, d = 4, 1_000
+    U = torch.zeros((n, d), dtype=torch.float32, device="cuda")
+    ctx = B.Brace(n, 1, d)
+    out = ctx.new_output()
+    assert ctx.reduce_scatter_step_status(1, U) == B.ERR_BAD_STEP        # round not started
+    assert ctx.consensus_status(out) == B.ERR_BAD_STEP
+    assert ctx.allgather_step_status(0, out) == B.ERR_BAD_STEP
+    assert ctx.reduce_scatter_step_status(0, U) == B.OK
+    assert ctx.reduce_scatter_step_status(2, U) == B.ERR_BAD_STEP        # skipped hop 1
+    assert ctx.reduce_scatter_step_status(n - 1, U) == B.ERR_BAD_STEP    # out of range
+    assert ctx.reduce_scatter_step_status(-1, U) == B.ERR_BAD_STEP
+    assert ctx.consensus_status(out) == B.ERR_BAD_STEP                   # reduce not finished
+    assert ctx.reduce_scatter_step_status(1, U) == B.OK
+    assert ctx.reduce_scatter_step_status(1, U) == B.ERR_BAD_STEP        # repeated hop
+    assert ctx.reduce_scatter_step_status(2, U) == B.OK
+    assert ctx.allgather_step_status(0, out) == B.ERR_BAD_STEP           # consensus first
+    assert ctx.consensus_status(out) == B.OK
+    assert ctx.consensus_status(out) == B.ERR_BAD_STEP
+    assert ctx.allgather_step_status(1, out) == B.ERR_BAD_STEP
+    for t in range(n - 1):
+        assert ctx.allgather_step_status(t, out) == B.OK
+    assert ctx.allgather_step_status(0, out) == B.ERR_BAD_STEP           # round is over
+    assert ctx.reduce_scatter_step_status(0, U) == B.OK                  # step 0 restarts at any time
+    assert ctx.reduce_scatter_step_status(0, U) == B.OK
+    lib = B.lib()
+    assert lib.brace_aggregate(ctx._ctx, None, d, out.data_ptr(), out.stride(0), None) == B.ERR_INVALID_ARG
+    assert lib.brace_aggregate(ctx._ctx, U.data_ptr(), d - 1, out.data_ptr(), out.stride(0), None) == B.ERR_INVALID_ARG
+    assert lib.brace_aggregate(ctx._ctx, U.data_ptr(), d, None, out.stride(0), None) == B.ERR_INVALID_ARG
+    assert lib.brace_aggregate(ctx._ctx, U.data_ptr(), d, out.data_ptr(), (d + 31) // 32 - 1, None) == B.ERR_INVALID_ARG
+    # attack argument checks
+    a = B.make_attack(B.ATTACK_GAUSSIAN, sigma=1.0)                       # noise missing
+    assert lib.brace_inject_attack(ctx._ctx, a, U.data_ptr(), d, U.data_ptr(), d, None) == B.ERR_INVALID_ARG
+    a = B.make_attack(B.ATTACK_SCALE_OWN, byz_ids=[n])                    # id out of range
+    assert lib.brace_inject_attack(ctx._ctx, a, U.data_ptr(), d, U.data_ptr(), d, None) == B.ERR_INVALID_ARG
+    a = B.make_attack(9)
+    assert lib.brace_inject_attack(ctx._ctx, a, U.data_ptr(), d, U.data_ptr(), d, None) == B.ERR_INVALID_ARG
+    ctx2 = B.Brace(n, 2, d)
+    a = B.make_attack(B.ATTACK_SCALE_OWN, byz_ids=[1, 1])                 # duplicate id
+    assert lib.brace_inject_attack(ctx2._ctx, a, U.data_ptr(), d, U.data_ptr(), d, None) == B.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert ctx.last_cuda_error() == 0
+    ctx.close()
+    ctx2.close()
+
+
+# ------------------------------------------------------------------ attack injection + whole pipeline
+def _np(t):
+    return None if t is None else t.cpu().numpy()
+
+
+@pytest.mark.parametrize("name,d", [("cfg1", 100_000), ("cfg2", 66_667), ("cfg3", 50_002), ("cfg4", 30_001),
+                                    ("cfg5", 80_000)])
+@pytest.mark.parametrize("ids", ["default", "scattered"])
+def test_attack_injection_and_pipeline(name, d, ids):
+    w = W.scaled(W.WORKLOADS[name], d)
+    H = W.honest_updates(w, 0, device="cuda")
+    noise, unif = W.attack_draws(w, 0, device="cuda")
+    byz = list(range(w.f)) if ids == "default" else sorted(
+        np.random.default_rng(w.n).choice(w.n, w.f, replace=False).tolist(), reverse=True)
+    atk = B.make_attack(w.attack, scale=w.scale, sigma=w.sigma, kappa=w.kappa, prob=w.prob,
+                        byz_ids=None if ids == "default" else byz, noise=noise, uniform=unif)
+    ctx = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam))
+    U = H.clone()
+    ctx.inject_attack(atk, H, U)                                           # separate source and destination
+    U2 = H.clone()
+    ctx.inject_attack(atk, U2, U2)                                         # in place
+    assert torch.equal(U, U2)
+    Hh = H.cpu().numpy()[:, :d]
+    exp = O.inject_attack(w.attack, Hh, byz, scale=w.scale, sigma=w.sigma, kappa=w.kappa, prob=w.prob,
+                          noise=None if noise is None else _np(noise)[:, :d],
+                          uniform=None if unif is None else _np(unif)[:, :d])
+    got = U.cpu().numpy()[:, :d]
+    denom = np.maximum(np.abs(exp), 1e-30)
+    assert (np.abs(got - exp) / denom).max() <= REL_TOL
+    assert np.array_equal(np.sign(got), np.sign(exp))                      # the votes are identical
+    assert np.array_equal(got.view(np.uint32), exp.view(np.uint32))        # and, by construction, the bits
+    assert torch.equal(U[:, d:], H[:, d:])                                 # padding untouched
+    # ring on the library's own injected matrix vs oracle on the oracle's
+    out = ctx.new_output()
+    ctx.aggregate(U, out)
+    tr = O.ring_round(exp, lam=w.lam, keep_states=False)
+    check_final(out, tr, B.RULE_SIGN_CONSENSUS, d)
+    assert np.array_equal(tr.outputs[0], O.gar_direct(exp, w.lam))
+    ctx.close()
+
+
+def test_host_buffer_round():
+    """brace_aggregate_host: pinned host in, host out, attack applied on the device copy."""
+    for name in ("cfg2", "cfg5", "cfg4"):
+        w = W.scaled(W.WORKLOADS[name], 20_001)
+        H = W.honest_updates(w, 0).pin_memory()
+        noise, unif = W.attack_draws(w, 0)
+        atk = B.make_attack(w.attack, scale=w.scale, sigma=w.sigma, kappa=w.kappa, prob=w.prob,
+                            noise=None if noise is None else noise.pin_memory(),
+                            uniform=None if unif is None else unif.pin_memory())
+        ctx = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam))
+        d_out = ctx.new_output()
+        h_out = torch.zeros(d_out.shape, dtype=d_out.dtype).pin_memory()
+        d_U = torch.empty(H.shape, dtype=torch.float32, device="cuda")
+        d_noise = None if noise is None else torch.empty(noise.shape, dtype=torch.float32, device="cuda")
+        d_unif = None if unif is None else torch.empty(unif.shape, dtype=torch.float32, device="cuda")
+        ctx.aggregate_host(atk, H, h_out, d_U, d_out, d_noise, d_unif)
+        torch.cuda.synchronize()
+        exp = O.inject_attack(w.attack, H.numpy()[:, :w.d], list(range(w.f)), scale=w.scale, sigma=w.sigma,
+                              kappa=w.kappa, prob=w.prob, noise=None if noise is None else noise.numpy()[:, :w.d],
+                              uniform=None if unif is None else unif.numpy()[:, :w.d])
+        tr = O.ring_round(exp, lam=w.lam, keep_states=False)
+        got = h_out[:, : (w.d + 31) // 32].numpy().view(np.uint32)
+        ew = expected_words(tr.outputs[0], w.d)
+        for c in range(w.n):
+            assert np.array_equal(got[c], ew)
+        ctx.close()
