@@ -219,6 +219,42 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
  * depend on either. */
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid);
 
+/* Bytes of mailbox scratch built into the library for brace_aggregate_static. */
+#define BRACE_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
+
+/* A whole round without a context and without a workspace (no counterpart in
+ * the paper: this is a packaging variant of brace_aggregate's fused kernel).
+ *
+ * Who needs it: code that may not obtain device memory at the point where it
+ * aggregates -- a plugin running inside a host application whose allocator owns
+ * all of HBM and offers no scratch to plugins, a service whose memory budget is
+ * frozen after start-up, a callback that runs where cudaMalloc is forbidden.
+ * Such callers still own their input and output buffers, but cannot size and
+ * allocate the mailbox workspace brace_init asks for.  Here the mailboxes live
+ * in a fixed array of BRACE_STATIC_SCRATCH_BYTES compiled into the library's
+ * device image (each GPU that loads the library keeps it until the process
+ * ends).  The call makes no cudaMalloc / cudaFree and calls no allocating
+ * routine; the context it uses internally lives on the host stack.
+ *
+ * Arguments as for brace_init (n, d, params; f is not needed) and
+ * brace_aggregate (d_updates [n][ld] float32, d_out [n][out_ld] packed uint32
+ * rows, or float32 rows for the sum rule).  Always runs the fused kernel, so it
+ * needs granule % 128 == 0, ld % 4 == 0 and 16-byte aligned d_updates (sum rule:
+ * also out_ld % 4 == 0 and aligned d_out); otherwise BRACE_ERR_UNSUPPORTED.
+ * Limit: 2 * round_up(n * round_up(longest sub-vector, 128) * entry bytes, 256)
+ * must not exceed BRACE_STATIC_SCRATCH_BYTES (about d <= 4.1 million for n <= 127
+ * under the sign rule, d <= 1.0 million under the sum rule); larger requests
+ * return BRACE_ERR_WORKSPACE and launch nothing.
+ *
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call outside any stream capture.  All calls
+ * on a device share the one array: it keeps whatever the previous call left
+ * (nothing in it has to start at zero -- the kernel only writes it), and two
+ * calls whose kernels may overlap on the GPU (different streams) race on it:
+ * serialise them.  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */
+int brace_aggregate_static(int32_t n, int64_t d, const brace_params* params, const float* d_updates,
+                           int64_t ld, void* d_out, int64_t out_ld, brace_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

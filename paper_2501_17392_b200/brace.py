@@ -62,7 +62,11 @@ SIGNATURES = {
     "brace_debug_mailbox": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_int64),
                                       C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
     "brace_set_tuning": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
+    "brace_aggregate_static": (C.c_int, [C.c_int32, C.c_int64, C.POINTER(Params), C.c_void_p, C.c_int64, C.c_void_p,
+                                         C.c_int64, C.c_void_p]),
 }
+
+STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
 def lib() -> C.CDLL:
@@ -130,6 +134,18 @@ def make_attack(kind: int, *, scale=1.0, sigma=1.0, kappa=3.0, prob=0.1, byz_ids
         a._uniform_keepalive = uniform
         a.uniform, a.uniform_ld = _ptr(uniform), uniform.stride(0)
     return a
+
+
+def aggregate_static_status(n: int, d: int, params: Params, updates: torch.Tensor, out: torch.Tensor,
+                            stream=None) -> int:
+    """brace_aggregate_static: a fused round whose mailboxes live in the library's
+    built-in scratch array, for callers that cannot allocate a workspace."""
+    return lib().brace_aggregate_static(n, d, C.byref(params), _ptr(updates), updates.stride(0), _ptr(out),
+                                        out.stride(0), _stream(stream))
+
+
+def aggregate_static(n: int, d: int, params: Params, updates: torch.Tensor, out: torch.Tensor, stream=None):
+    _check(aggregate_static_status(n, d, params, updates, out, stream), "brace_aggregate_static")
 
 
 class Brace:

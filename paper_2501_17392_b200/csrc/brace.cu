@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -385,6 +386,40 @@ int aggregate_impl(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_
 
 }  // namespace
 
+// ---- round without a caller workspace ---------------------------------------------------------
+// Mailbox scratch for brace_aggregate_static.  Every GPU that loads the library
+// holds these bytes until the process exits.  In host code the symbol's name is
+// only a handle: the device address is fetched once per device with
+// cudaGetSymbolAddress and that pointer is what the kernels receive.
+constexpr size_t kStaticScratchBytes = (size_t)BRACE_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {nullptr};
+
+// Device address of g_static_scratch on the current device (looked up on first use).
+cudaError_t static_scratch_for_current_device(void** out) {
+  int dev = -1;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[dev]) {
+    void* ptr = nullptr;
+    err = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (err != cudaSuccess) return err;
+    if (!ptr || (reinterpret_cast<uintptr_t>(ptr) & 255u) != 0) return cudaErrorInvalidSymbol;
+    g_static_ptr[dev] = ptr;
+  }
+  *out = g_static_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+
 // =============================================================================================
 // C ABI
 // =============================================================================================
@@ -625,6 +660,48 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
   if (segment) *segment = j;
   if (entry_bytes) *entry_bytes = ctx->entry_bytes;
   return BRACE_OK;
+}
+
+int brace_aggregate_static(int32_t n, int64_t d, const brace_params* params, const float* d_updates, int64_t ld,
+                           void* d_out, int64_t out_ld, brace_stream_t stream) {
+  if (n < 2 || d < 1 || !params_ok(params)) return BRACE_ERR_INVALID_ARG;
+  const int eb = entry_bytes_for(n, params->rule);
+  if (eb == 0) return BRACE_ERR_UNSUPPORTED;
+  // size check first: a request that cannot fit is refused before any CUDA call
+  const Part pt = make_part(n, d, params->granule);
+  const int64_t seg_max = longest_segment(pt);
+  const int64_t seg_pad = round_up(seg_max > 0 ? seg_max : 1, kMailAlign);
+  const size_t one_set = (size_t)round_up((int64_t)n * seg_pad * eb, 256);
+  if (2 * one_set > kStaticScratchBytes) return BRACE_ERR_WORKSPACE;
+
+  brace_ctx ctx;                       // host stack only; its vectors stay empty
+  ctx.n = n;
+  ctx.f = 0;
+  ctx.d = d;
+  ctx.p = *params;
+  ctx.pt = pt;
+  double fl = std::floor((double)params->lambda);
+  if (fl < -(double)n - 1.0) fl = -(double)n - 1.0;
+  if (fl > (double)n) fl = (double)n;
+  ctx.lam_i = (int)fl;
+  ctx.entry_bytes = eb;
+  ctx.seg_max = seg_max;
+  ctx.seg_pad = seg_pad;
+  int rc = check_updates(&ctx, d_updates, ld);
+  if (rc != BRACE_OK) return rc;
+  rc = check_out(&ctx, d_out, out_ld);
+  if (rc != BRACE_OK) return rc;
+  if (!fused_layout_ok(&ctx, d_updates, ld, d_out, out_ld)) return BRACE_ERR_UNSUPPORTED;
+  void* scratch = nullptr;
+  cudaError_t err = static_scratch_for_current_device(&scratch);
+  if (err != cudaSuccess) return BRACE_ERR_CUDA;
+  ctx.ws = static_cast<char*>(scratch);
+  ctx.ws_bytes = kStaticScratchBytes;
+  ctx.mail[0] = ctx.ws;
+  ctx.mail[1] = ctx.ws + one_set;
+  // nothing in the scratch has to start at zero: the fused kernel only writes the
+  // mailboxes (the partial sums travel in registers), so stale contents are harmless
+  return launch_fused(&ctx, d_updates, ld, d_out, out_ld, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"
