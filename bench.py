@@ -378,6 +378,7 @@ def main():
     ap.add_argument("--mode", default="fused", choices=["fused", "stepwise", "auto"])
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--grid", type=int, default=0)
+    ap.add_argument("--d", type=int, default=0, help="override the workload's vector length (profiling on a small case)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -386,6 +387,8 @@ def main():
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
     w = W.WORKLOADS[args.workload]
+    if args.d:
+        w = W.scaled(w, args.d)
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -51,6 +51,8 @@ struct brace_ctx {
   // launch tuning (0 = default)
   int fused_variant = 0;
   int fused_grid = 0;
+  int step_vpt = 0;
+  int stats_vw = 0;
 };
 
 namespace {
@@ -130,27 +132,42 @@ int launch_rs_step(brace_ctx* ctx, int step, const float* U, int64_t ld, cudaStr
   const int n = ctx->n;
   const int in_set = step & 1, out_set = (step + 1) & 1;
   const bool vec = vec_layout_ok(ctx, U, ld);
-  const int64_t per_block = vec ? kThreads * 4 : kThreads;
+  // float4 per thread: enough loads in flight for long sub-vectors, enough CTAs for short ones
+  int vpt = 0;
+  if (vec) {
+    vpt = ctx->step_vpt > 0 ? ctx->step_vpt : 4;
+    while (vpt > 1 && (int64_t)n * ((ctx->seg_max + 1024 * vpt - 1) / (1024 * vpt)) < 4 * kSmCount) vpt >>= 1;
+  }
+  const int64_t per_block = vec ? (int64_t)kThreads * 4 * vpt : kThreads;
   dim3 grid(tiles(ctx->seg_max, per_block), (unsigned)n);
   const bool zs = ctx->p.zero_sign != 0;
   const int zsv = ctx->p.zero_sign;
-#define BRACE_RS_SIGN(P, VEC, ZS)                                                                            \
-  rs_step_sign_kernel<P, VEC, ZS><<<grid, kThreads, 0, st>>>(ctx->pt, U, ld, (const P*)ctx->mail[in_set],    \
+#define BRACE_RS_SIGN(P, VPT, ZS)                                                                            \
+  rs_step_sign_kernel<P, VPT, ZS><<<grid, kThreads, 0, st>>>(ctx->pt, U, ld, (const P*)ctx->mail[in_set],    \
                                                              (P*)ctx->mail[out_set], ctx->seg_pad, step, zsv)
+#define BRACE_RS_SIGN_P(P)                                                                         \
+  do {                                                                                             \
+    switch (vpt) {                                                                                 \
+      case 4: if (zs) BRACE_RS_SIGN(P, 4, true); else BRACE_RS_SIGN(P, 4, false); break;           \
+      case 2: if (zs) BRACE_RS_SIGN(P, 2, true); else BRACE_RS_SIGN(P, 2, false); break;           \
+      case 1: if (zs) BRACE_RS_SIGN(P, 1, true); else BRACE_RS_SIGN(P, 1, false); break;           \
+      default: if (zs) BRACE_RS_SIGN(P, 0, true); else BRACE_RS_SIGN(P, 0, false); break;          \
+    }                                                                                              \
+  } while (0)
   if (ctx->p.rule == BRACE_RULE_SUM) {
+    dim3 gsum(tiles(ctx->seg_max, vec ? kThreads * 4 : kThreads), (unsigned)n);
     if (vec)
-      rs_step_sum_kernel<true><<<grid, kThreads, 0, st>>>(ctx->pt, U, ld, (const float*)ctx->mail[in_set],
+      rs_step_sum_kernel<true><<<gsum, kThreads, 0, st>>>(ctx->pt, U, ld, (const float*)ctx->mail[in_set],
                                                           (float*)ctx->mail[out_set], ctx->seg_pad, step);
     else
-      rs_step_sum_kernel<false><<<grid, kThreads, 0, st>>>(ctx->pt, U, ld, (const float*)ctx->mail[in_set],
+      rs_step_sum_kernel<false><<<gsum, kThreads, 0, st>>>(ctx->pt, U, ld, (const float*)ctx->mail[in_set],
                                                            (float*)ctx->mail[out_set], ctx->seg_pad, step);
   } else if (ctx->entry_bytes == 1) {
-    if (vec) { if (zs) BRACE_RS_SIGN(int8_t, true, true); else BRACE_RS_SIGN(int8_t, true, false); }
-    else     { if (zs) BRACE_RS_SIGN(int8_t, false, true); else BRACE_RS_SIGN(int8_t, false, false); }
+    BRACE_RS_SIGN_P(int8_t);
   } else {
-    if (vec) { if (zs) BRACE_RS_SIGN(int16_t, true, true); else BRACE_RS_SIGN(int16_t, true, false); }
-    else     { if (zs) BRACE_RS_SIGN(int16_t, false, true); else BRACE_RS_SIGN(int16_t, false, false); }
+    BRACE_RS_SIGN_P(int16_t);
   }
+#undef BRACE_RS_SIGN_P
 #undef BRACE_RS_SIGN
   return check_launch(ctx);
 }
@@ -346,19 +363,55 @@ int inject_impl(brace_ctx* ctx, const brace_attack* atk, const float* H, int64_t
   if (kind == BRACE_ATTACK_SPARSE_NOISE && (!atk->uniform || atk->uniform_ld < ctx->d)) return BRACE_ERR_INVALID_ARG;
   int rc = stage_ids(ctx, atk->h_byz_ids, st);
   if (rc != BRACE_OK) return rc;
+  const bool rows16 = (ld_h % 4 == 0) && (ld_u % 4 == 0) && aligned16(H) && aligned16(Uo);
   if (kind == BRACE_ATTACK_SCALED_MEAN || kind == BRACE_ATTACK_MEAN_SHIFT) {
-    // two passes over the honest rows: keep the set of coordinates in flight small
-    // enough that the second pass finds the first one's lines in L2
-    int64_t blocks = (ctx->d + kThreads - 1) / kThreads;
-    const int64_t cap = (int64_t)kSmCount * 4;
-    if (blocks > cap) blocks = cap;
-    inject_stats_kernel<8><<<(unsigned)blocks, kThreads, 0, st>>>(kind, ctx->d_ids, ctx->f, ctx->n, H, ld_h, Uo, ld_u,
-                                                                 ctx->d, atk->scale, atk->kappa);
+    const int m = ctx->n - ctx->f;
+    const int mpad = (m + 7) / 8 * 8;
+    // staged variant: one column (vw floats wide) of all m honest rows per thread in shared memory
+    const bool rows8 = (ld_h % 2 == 0) && (ld_u % 2 == 0) && (reinterpret_cast<uintptr_t>(H) & 7u) == 0 &&
+                       (reinterpret_cast<uintptr_t>(Uo) & 7u) == 0;
+    int vw = ctx->stats_vw > 0 ? ctx->stats_vw : 2;
+    if (vw == 4 && !rows16) vw = 2;
+    if (vw == 2 && !rows8) vw = 1;
+    const bool layout_ok = true;
+    int T = 1024 / vw;
+    while (T > 32 && (size_t)mpad * T * vw * 4 > 40 * 1024) T >>= 1;
+    const size_t smem = (size_t)mpad * T * vw * 4 + (size_t)mpad * 8;
+    if (layout_ok && smem <= 200 * 1024) {
+      auto kern = vw == 1 ? inject_stats_smem_kernel<1, 12>
+                          : (vw == 2 ? inject_stats_smem_kernel<2, 12> : inject_stats_smem_kernel<4, 12>);
+      if (smem > 48 * 1024) {
+        cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return cuda_fail(ctx, err);
+      }
+      int64_t blocks = (ctx->d + (int64_t)T * vw - 1) / ((int64_t)T * vw);
+      const int64_t cap = (int64_t)kSmCount * 64;
+      if (blocks > cap) blocks = cap;
+      kern<<<(unsigned)blocks, T, smem, st>>>(kind, ctx->d_ids, ctx->f, ctx->n, H, ld_h, Uo, ld_u, ctx->d,
+                                             atk->scale, atk->kappa);
+    } else {
+      // two passes over the honest rows in global memory: keep the set of coordinates in
+      // flight small enough that the second pass finds the first one's lines in L2
+      int64_t blocks = (ctx->d + kThreads - 1) / kThreads;
+      const int64_t cap = (int64_t)kSmCount * 4;
+      if (blocks > cap) blocks = cap;
+      inject_stats_kernel<8><<<(unsigned)blocks, kThreads, 0, st>>>(kind, ctx->d_ids, ctx->f, ctx->n, H, ld_h, Uo,
+                                                                   ld_u, ctx->d, atk->scale, atk->kappa);
+    }
   } else {
-    dim3 grid(tiles(ctx->d, kThreads), (unsigned)ctx->f);
-    inject_elementwise_kernel<<<grid, kThreads, 0, st>>>(kind, ctx->d_ids, H, ld_h, Uo, ld_u, atk->noise,
-                                                        atk->noise_ld, atk->uniform, atk->uniform_ld, ctx->d,
-                                                        atk->scale, atk->sigma, atk->prob);
+    const bool draws16 = (!needs_noise || (atk->noise_ld % 4 == 0 && aligned16(atk->noise))) &&
+                         (kind != BRACE_ATTACK_SPARSE_NOISE || (atk->uniform_ld % 4 == 0 && aligned16(atk->uniform)));
+    if (rows16 && draws16) {
+      dim3 grid(tiles(ctx->d, kThreads * 4), (unsigned)ctx->f);
+      inject_elementwise_vec_kernel<<<grid, kThreads, 0, st>>>(kind, ctx->d_ids, H, ld_h, Uo, ld_u, atk->noise,
+                                                              atk->noise_ld, atk->uniform, atk->uniform_ld, ctx->d,
+                                                              atk->scale, atk->sigma, atk->prob);
+    } else {
+      dim3 grid(tiles(ctx->d, kThreads), (unsigned)ctx->f);
+      inject_elementwise_kernel<<<grid, kThreads, 0, st>>>(kind, ctx->d_ids, H, ld_h, Uo, ld_u, atk->noise,
+                                                          atk->noise_ld, atk->uniform, atk->uniform_ld, ctx->d,
+                                                          atk->scale, atk->sigma, atk->prob);
+    }
   }
   return check_launch(ctx);
 }
@@ -509,7 +562,15 @@ int brace_segment(const brace_ctx* ctx, int32_t j, int64_t* begin, int64_t* end)
 int brace_last_cuda_error(const brace_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
 
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid) {
-  if (!ctx || fused_variant < 0 || fused_variant > 5 || fused_grid < 0) return BRACE_ERR_INVALID_ARG;
+  if (!ctx || fused_variant < 0 || fused_grid < 0) return BRACE_ERR_INVALID_ARG;
+  const int stats_code = fused_variant / 100;    // hundreds digit: floats per thread of the statistics kernel
+  const int step_code = (fused_variant / 10) % 10;   // tens digit: float4 per thread of the hop kernel
+  fused_variant %= 10;
+  if (fused_variant > 5 || (step_code != 0 && step_code != 1 && step_code != 2 && step_code != 4) ||
+      (stats_code != 0 && stats_code != 1 && stats_code != 2 && stats_code != 4))
+    return BRACE_ERR_INVALID_ARG;
+  ctx->step_vpt = step_code;
+  ctx->stats_vw = stats_code;
   ctx->fused_variant = fused_variant;
   ctx->fused_grid = fused_grid;
   return BRACE_OK;

@@ -55,9 +55,11 @@ __device__ __forceinline__ void load4(const int16_t* p, int& a, int& b, int& c, 
 
 // ---------------------------------------------------------------------------
 // Share-Reduce hop, sign rule (Section 3 Phase II; Phase I fused into the read).
-// grid = (tiles over the longest sub-vector, n senders); one float4 per thread.
+// grid = (tiles over the longest sub-vector, n senders).  Vector variant: a CTA
+// covers 256*VPT float4; every thread issues its VPT update loads (and mailbox
+// loads) before it consumes any of them.
 // ---------------------------------------------------------------------------
-template <typename P, bool VEC, bool ZS>
+template <typename P, int VPT, bool ZS>
 __global__ void __launch_bounds__(256)
 rs_step_sign_kernel(Part pt, const float* __restrict__ U, int64_t ld, const P* __restrict__ mail_in,
                     P* __restrict__ mail_out, int64_t seg_pad, int step, int zs) {
@@ -72,30 +74,45 @@ rs_step_sign_kernel(Part pt, const float* __restrict__ U, int64_t ld, const P* _
   const float* ur = U + (int64_t)r * ld + b;
   const P* in = mail_in + (int64_t)c * seg_pad;
   P* out = mail_out + (int64_t)r * seg_pad;
-  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (VEC) {
-    const int64_t i = t * 4;
-    if (i + 4 <= L) {
-      float4 x = ld_stream(ur + i);
-      int a0, a1, a2, a3;
-      if (step == 0) {
-        float4 y = ld_stream(uc + i);
-        a0 = sgn1<ZS>(y.x, zs); a1 = sgn1<ZS>(y.y, zs); a2 = sgn1<ZS>(y.z, zs); a3 = sgn1<ZS>(y.w, zs);
-      } else {
-        load4(in + i, a0, a1, a2, a3);
+  if (VPT > 0) {
+    constexpr int V = VPT > 0 ? VPT : 1;
+    const int64_t base = (int64_t)blockIdx.x * (256 * V) + threadIdx.x;
+    if (base * 4 >= L) return;
+    float4 x[V], y[V];
+    int a[V][4];
+    bool full[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      const int64_t i = (base + v * 256) * 4;
+      full[v] = i + 4 <= L;
+      if (full[v]) {
+        x[v] = ld_stream(ur + i);
+        if (step == 0) y[v] = ld_stream(uc + i);
+        else load4(in + i, a[v][0], a[v][1], a[v][2], a[v][3]);
       }
-      store4(out + i, a0 + sgn1<ZS>(x.x, zs), a1 + sgn1<ZS>(x.y, zs), a2 + sgn1<ZS>(x.z, zs),
-             a3 + sgn1<ZS>(x.w, zs));
-    } else {
-      for (int64_t k = i; k < L; ++k) {
-        int a = (step == 0) ? sgn1<ZS>(uc[k], zs) : (int)in[k];
-        out[k] = (P)(a + sgn1<ZS>(ur[k], zs));
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      const int64_t i = (base + v * 256) * 4;
+      if (full[v]) {
+        if (step == 0) {
+          a[v][0] = sgn1<ZS>(y[v].x, zs); a[v][1] = sgn1<ZS>(y[v].y, zs);
+          a[v][2] = sgn1<ZS>(y[v].z, zs); a[v][3] = sgn1<ZS>(y[v].w, zs);
+        }
+        store4(out + i, a[v][0] + sgn1<ZS>(x[v].x, zs), a[v][1] + sgn1<ZS>(x[v].y, zs),
+               a[v][2] + sgn1<ZS>(x[v].z, zs), a[v][3] + sgn1<ZS>(x[v].w, zs));
+      } else {
+        for (int64_t k = i; k < L; ++k) {         // ragged end of the last sub-vector
+          const int s0 = (step == 0) ? sgn1<ZS>(uc[k], zs) : (int)in[k];
+          out[k] = (P)(s0 + sgn1<ZS>(ur[k], zs));
+        }
       }
     }
   } else {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t < L) {
-      int a = (step == 0) ? sgn1<ZS>(uc[t], zs) : (int)in[t];
-      out[t] = (P)(a + sgn1<ZS>(ur[t], zs));
+      int s0 = (step == 0) ? sgn1<ZS>(uc[t], zs) : (int)in[t];
+      out[t] = (P)(s0 + sgn1<ZS>(ur[t], zs));
     }
   }
 }
@@ -558,6 +575,169 @@ inject_stats_kernel(int kind, const int* __restrict__ ids, int f, int n, const f
     }
     const float v = __double2float_rn(vec);
     for (int bq = 0; bq < f; ++bq) Uo[(int64_t)ids[bq] * ld_u + k] = v;
+  }
+}
+
+
+// 128-bit variant of the element-wise alterations (rows 16-byte aligned).
+__global__ void __launch_bounds__(256)
+inject_elementwise_vec_kernel(int kind, const int* __restrict__ ids, const float* H, int64_t ld_h, float* Uo,
+                              int64_t ld_u, const float* __restrict__ noise, int64_t ld_z,
+                              const float* __restrict__ unif, int64_t ld_r, int64_t d, float scale, float sigma,
+                              float prob) {
+  const int bidx = blockIdx.y;
+  const int id = ids[bidx];
+  const int64_t k = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (k >= d) return;
+  float4 v;
+  if (kind == 1) {
+    const float4 h = *reinterpret_cast<const float4*>(H + (int64_t)id * ld_h + k);
+    v = make_float4(__fmul_rn(scale, h.x), __fmul_rn(scale, h.y), __fmul_rn(scale, h.z), __fmul_rn(scale, h.w));
+  } else {
+    const float4 z = ld_stream(noise + (int64_t)bidx * ld_z + k);
+    v = make_float4(__fmul_rn(sigma, z.x), __fmul_rn(sigma, z.y), __fmul_rn(sigma, z.z), __fmul_rn(sigma, z.w));
+    if (kind != 2) {
+      const float4 u = ld_stream(unif + (int64_t)bidx * ld_r + k);
+      v.x = (u.x < prob) ? v.x : 0.0f;
+      v.y = (u.y < prob) ? v.y : 0.0f;
+      v.z = (u.z < prob) ? v.z : 0.0f;
+      v.w = (u.w < prob) ? v.w : 0.0f;
+    }
+  }
+  float* dst = Uo + (int64_t)id * ld_u + k;
+  if (k + 4 <= d) {
+    *reinterpret_cast<float4*>(dst) = v;
+  } else {                                          // ragged end: never write past coordinate d-1
+    const float t[4] = {v.x, v.y, v.z, v.w};
+    for (int q = 0; k + q < d; ++q) dst[q] = t[q];
+  }
+}
+
+// Mean / mean-shift alterations with the honest rows of a tile staged in shared
+// memory by asynchronous 16-byte copies: the rows of the tile are requested far
+// ahead of their use (many loads in flight without holding registers), the
+// float64 sum consumes them eight rows at a time as they land, and the second
+// pass (deviations) re-reads shared memory instead of HBM.  Each thread owns one
+// float4 column of the tile, so no barrier is needed after the row offsets are
+// published.  Arithmetic and order are those of inject_stats_kernel.
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+  const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+template <int VW> struct StageVec;
+template <> struct StageVec<1> { typedef float type; };
+template <> struct StageVec<2> { typedef float2 type; };
+template <> struct StageVec<4> { typedef float4 type; };
+
+template <int VW>
+__device__ __forceinline__ void cp_async_vw(void* smem, const void* gmem) {
+  const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+  if (VW == 4) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem));
+  else if (VW == 2) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(s), "l"(gmem));
+  else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(s), "l"(gmem));
+}
+
+// VW = floats per thread (1, 2 or 4): fewer floats per thread means more warps
+// for the same shared-memory tile.
+template <int VW, int DEPTH>
+__global__ void inject_stats_smem_kernel(int kind, const int* __restrict__ ids, int f, int n, const float* H,
+                                         int64_t ld_h, float* Uo, int64_t ld_u, int64_t d, float scale,
+                                         float kappa) {
+  constexpr int GROUP = 8;
+  typedef typename StageVec<VW>::type V;
+  extern __shared__ float4 sm_raw[];                // [mpad][blockDim.x] columns of V, then mpad row offsets
+  V* sm_rows = reinterpret_cast<V*>(sm_raw);
+  const int m = n - f;
+  const int ngroups = (m + GROUP - 1) / GROUP;
+  const int mpad = ngroups * GROUP;
+  const int T = blockDim.x, tid = threadIdx.x;
+  int64_t* rowoff = reinterpret_cast<int64_t*>(sm_rows + (size_t)mpad * T);
+  for (int r = tid; r < mpad; r += T) rowoff[r] = (int64_t)ids[f + (r < m ? r : m - 1)] * ld_h;
+  __syncthreads();
+  const int64_t ntiles = (d + (int64_t)T * VW - 1) / ((int64_t)T * VW);
+  V* col = sm_rows + tid;
+  for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    const int64_t k = (tile * T + tid) * VW;
+    const bool active = k < d;
+    const float* src = H + k;
+    auto issue = [&](int g) {
+      if (active && g < ngroups) {
+#pragma unroll
+        for (int q = 0; q < GROUP; ++q) {
+          const int r = g * GROUP + q;
+          if (r < m) cp_async_vw<VW>(col + (size_t)r * T, src + rowoff[r]);
+        }
+      }
+      cp_async_commit();
+    };
+#pragma unroll 1
+    for (int g = 0; g < DEPTH; ++g) issue(g);
+    double tot[VW];
+#pragma unroll
+    for (int e = 0; e < VW; ++e) tot[e] = 0.0;
+#pragma unroll 1
+    for (int g = 0; g < ngroups; ++g) {
+      cp_async_wait<DEPTH - 1>();
+      if (active) {
+        V x[GROUP];
+#pragma unroll
+        for (int q = 0; q < GROUP; ++q) x[q] = col[(size_t)(g * GROUP + q) * T];
+#pragma unroll
+        for (int q = 0; q < GROUP; ++q) {
+          if (g * GROUP + q < m) {
+            const float* xe = reinterpret_cast<const float*>(&x[q]);
+#pragma unroll
+            for (int e = 0; e < VW; ++e) tot[e] = __dadd_rn(tot[e], (double)xe[e]);
+          }
+        }
+      }
+      issue(g + DEPTH);
+    }
+    cp_async_wait<0>();
+    if (!active) continue;
+    double vec[VW];
+    const double dm = (double)m;
+    if (kind == 3) {
+#pragma unroll
+      for (int e = 0; e < VW; ++e) vec[e] = __dmul_rn((double)scale, __ddiv_rn(tot[e], dm));
+    } else {
+      double mean[VW], sq[VW];
+#pragma unroll
+      for (int e = 0; e < VW; ++e) { mean[e] = __ddiv_rn(tot[e], dm); sq[e] = 0.0; }
+#pragma unroll 1
+      for (int g = 0; g < ngroups; ++g) {
+        V x[GROUP];
+#pragma unroll
+        for (int q = 0; q < GROUP; ++q) x[q] = col[(size_t)(g * GROUP + q) * T];
+#pragma unroll
+        for (int q = 0; q < GROUP; ++q) {
+          if (g * GROUP + q < m) {
+            const float* xe = reinterpret_cast<const float*>(&x[q]);
+#pragma unroll
+            for (int e = 0; e < VW; ++e) {
+              const double dev = __dsub_rn((double)xe[e], mean[e]);
+              sq[e] = __dadd_rn(sq[e], __dmul_rn(dev, dev));
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < VW; ++e)
+        vec[e] = __dsub_rn(mean[e], __dmul_rn((double)kappa, __dsqrt_rn(__ddiv_rn(sq[e], dm))));
+    }
+    float t[VW];
+#pragma unroll
+    for (int e = 0; e < VW; ++e) t[e] = __double2float_rn(vec[e]);
+    if (k + VW <= d) {
+      for (int bq = 0; bq < f; ++bq) *reinterpret_cast<V*>(Uo + (int64_t)ids[bq] * ld_u + k) = *reinterpret_cast<V*>(t);
+    } else {
+      for (int bq = 0; bq < f; ++bq)
+        for (int e = 0; k + e < d; ++e) Uo[(int64_t)ids[bq] * ld_u + k + e] = t[e];
+    }
   }
 }
 

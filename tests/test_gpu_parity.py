@@ -164,6 +164,14 @@ def test_hop_by_hop_and_whole_round(n, d, G, ld, lam, zs, rule):
     out2 = torch.full_like(out, 5)
     ctx.aggregate(Ud, out2)
     check_final(out2, tr, rule, d)
+    for code in (10, 20, 40):                           # hop kernel with 1 / 2 / 4 float4 per thread
+        ctx.set_tuning(code, 0)
+        out2.fill_(5)
+        ctx.aggregate(Ud, out2)
+        check_final(out2, tr, rule, d)
+        for c in range(n):
+            assert torch.equal(ctx.mailbox_tensor(c)[1], boxes_steps[0][c][1])
+    ctx.set_tuning(0, 0)
 
     # (3) whole round, fused kernel, every shape; mailboxes end as the step calls left them
     if fusable:
@@ -403,6 +411,26 @@ def test_attack_injection_and_pipeline(name, d, ids):
     tr = O.ring_round(exp, lam=w.lam, keep_states=False)
     check_final(out, tr, B.RULE_SIGN_CONSENSUS, d)
     assert np.array_equal(tr.outputs[0], O.gar_direct(exp, w.lam))
+    ctx.close()
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+def test_attack_injection_unaligned_rows(name):
+    """Row strides that are not multiples of 4 take the scalar kernels; same bits."""
+    d, ld = 20_003, 20_005
+    w = W.scaled(W.WORKLOADS[name], d)
+    H = W.honest_updates(w, 1, device="cuda", ld=ld)
+    noise, unif = W.attack_draws(w, 1, device="cuda", ld=ld + 2)
+    atk = B.make_attack(w.attack, scale=w.scale, sigma=w.sigma, kappa=w.kappa, prob=w.prob, noise=noise, uniform=unif)
+    ctx = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam))
+    U = H.clone()
+    ctx.inject_attack(atk, H, U)
+    exp = O.inject_attack(w.attack, H.cpu().numpy()[:, :d], list(range(w.f)), scale=w.scale, sigma=w.sigma,
+                          kappa=w.kappa, prob=w.prob, noise=None if noise is None else _np(noise)[:, :d],
+                          uniform=None if unif is None else _np(unif)[:, :d])
+    got = U.cpu().numpy()
+    assert np.array_equal(got[:, :d].view(np.uint32), exp.view(np.uint32))
+    assert torch.equal(U[:, d:], H[:, d:])
     ctx.close()
 
 
