@@ -119,6 +119,11 @@ def max_over_ranks(value: float, world: int, device) -> float:
     return float(t.item())
 
 
+def whole_job_value(world: int, n: int, d: int, steps: int, total_ms: float) -> float:
+    """Elements all replicas aggregated, divided by the slowest rank's time."""
+    return world * n * d * steps / (total_ms * 1e-3)
+
+
 def algorithmic_bytes_fused(n: int, d: int, entry_bytes: int) -> int:
     """Bytes the fused round must move: every update read once, the last two hops'
     partials written to the mailboxes, every client's packed row written once."""
@@ -280,7 +285,7 @@ def run_cuda(args, w):
         e2e_ms = max_over_ranks(float(e0.elapsed_time(e1)), world, device)
         h2d = 4 * n * w.ld + (0 if noise is None else noise.numel() * 4) + (0 if unif is None else unif.numel() * 4)
         d2h = out.numel() * 4
-        e2e = {"value": world * n * d * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": whole_job_value(world, n, d, e2e_steps, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps}
         same = bool(torch.equal(h_out.to(device), out_ref))
         e2e["matches_device_result"] = same
@@ -344,7 +349,7 @@ def run_cuda(args, w):
                                   f"({dt:.1f} s)"}
 
     line = {
-        "metric": METRIC, "value": world * n * d * args.steps / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": whole_job_value(world, n, d, args.steps, total_ms), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32 sign-sums over f32 inputs", "data": "synthetic",
         "config": {"workload": w.name, "n": n, "f": f, "d": d, "lambda": w.lam, "rounds_per_step": 1,

@@ -135,7 +135,7 @@ int launch_rs_step(brace_ctx* ctx, int step, const float* U, int64_t ld, cudaStr
   // float4 per thread: enough loads in flight for long sub-vectors, enough CTAs for short ones
   int vpt = 0;
   if (vec) {
-    vpt = ctx->step_vpt > 0 ? ctx->step_vpt : 4;
+    vpt = ctx->step_vpt > 0 ? ctx->step_vpt : 2;
     while (vpt > 1 && (int64_t)n * ((ctx->seg_max + 1024 * vpt - 1) / (1024 * vpt)) < 4 * kSmCount) vpt >>= 1;
   }
   const int64_t per_block = vec ? (int64_t)kThreads * 4 * vpt : kThreads;

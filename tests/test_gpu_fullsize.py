@@ -1,0 +1,147 @@
+"""Parity at the full sizes of the five workloads, in the launch configuration
+bench.py times (fused round, default tuning; injection in its default kernels).
+
+The oracle cannot run 2.5e9 elements in test time, so the comparison is on
+sampled coordinates it computes one by one (Eq. (1) per coordinate needs only
+that coordinate's column): the head and the ragged tail of the vector, both
+sides of sub-vector boundaries, and random coordinates.  Properties that hold
+at any size are checked on the whole result: every client's row is identical,
+padding bits are zero, the hop-by-hop path leaves the same bits and mailboxes."""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import brace_oracle as O
+from paper_2501_17392_b200 import brace as B
+from paper_2501_17392_b200 import build as brace_build
+from paper_2501_17392_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    brace_build.build()
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+
+
+def sample_coordinates(ctx: B.Brace, d: int, n: int, seed: int) -> np.ndarray:
+    rng = np.random.default_rng(seed)
+    picks = [np.arange(0, min(d, 2048)), np.arange(max(0, d - 2048), d), rng.integers(0, d, size=8192)]
+    for j in sorted(set([0, 1, n // 2, n - 2, n - 1])):
+        b, e = ctx.segment(j)
+        picks.append(np.arange(max(0, b - 64), min(d, b + 64)))
+        picks.append(np.arange(max(0, e - 64), min(d, e + 64)))
+    return np.unique(np.concatenate(picks)).astype(np.int64)
+
+
+def bits_at(row_words: torch.Tensor, idx: torch.Tensor) -> np.ndarray:
+    w = row_words[idx // 32].to(torch.int64) & 0xFFFFFFFF
+    return ((w >> (idx % 32)) & 1).cpu().numpy().astype(np.int8)
+
+
+def one_round(w, ctx, H, noise, unif, rnd):
+    d, n = w.d, w.n
+    idx_np = sample_coordinates(ctx, d, n, seed=rnd + n)
+    idx = torch.as_tensor(idx_np, device="cuda")
+    Hs = H[:, idx].cpu().numpy()
+    atk = B.make_attack(w.attack, scale=w.scale, sigma=w.sigma, kappa=w.kappa, prob=w.prob, noise=noise, uniform=unif)
+    ctx.inject_attack(atk, H, H)                       # in place, as a Byzantine client would
+    U = H
+    Us = U[:, idx].cpu().numpy()
+    exp_u = O.inject_attack(w.attack, Hs, list(range(w.f)), scale=w.scale, sigma=w.sigma, kappa=w.kappa, prob=w.prob,
+                            noise=None if noise is None else noise[:, idx].cpu().numpy(),
+                            uniform=None if unif is None else unif[:, idx].cpu().numpy())
+    rel = np.abs(Us - exp_u) / np.maximum(np.abs(exp_u), 1e-30)
+    assert rel.max() <= 1e-5
+    assert np.array_equal(Us.view(np.uint32), exp_u.view(np.uint32))
+
+    out = ctx.new_output()
+    out.fill_(-1)
+    ctx.aggregate(U, out)
+    torch.cuda.synchronize()
+    words = (d + 31) // 32
+    # any-size properties
+    for c in range(1, n):
+        assert torch.equal(out[c, :words], out[0, :words]), f"client {c} differs from client 0"
+    if d % 32:
+        last = int(out[0, words - 1].item()) & 0xFFFFFFFF
+        assert last >> (d % 32) == 0, "padding bits must be zero"
+    # sampled coordinates against Eq. (1)
+    exp_bits = (O.gar_direct(exp_u, w.lam) > 0).astype(np.int8)
+    assert np.array_equal(bits_at(out[0], idx), exp_bits)
+    # the owners' final partial sign-sums at the sampled coordinates
+    S = O.sign_sum_direct(exp_u)
+    for j in sorted(set([0, 1, n // 2, n - 1])):
+        owner = (j - 1) % n
+        b, e = ctx.segment(j)
+        seg, box = ctx.mailbox_tensor(owner)
+        assert seg == j and box.numel() == e - b
+        sel = (idx_np >= b) & (idx_np < e)
+        assert np.array_equal(box.numpy()[idx_np[sel] - b].astype(np.int32), S[sel])
+    return out, U
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
+def test_full_size_workload(name):
+    w = W.WORKLOADS[name]
+    ctx = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam, agg_mode=B.AGG_FUSED))
+    H = torch.zeros((w.n, w.ld), dtype=torch.float32, device="cuda")
+    out = U = None
+    for rnd in range(w.rounds):
+        W.honest_updates(w, rnd, device="cuda", out=H)
+        noise, unif = W.attack_draws(w, rnd, device="cuda")
+        out, U = one_round(w, ctx, H, noise, unif, rnd)
+        del noise, unif
+    # the hop-by-hop path on the same (last) inputs: same bits, same surviving mailboxes
+    ctx_s = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam, agg_mode=B.AGG_STEPWISE))
+    out_s = ctx_s.new_output()
+    ctx_s.aggregate(U, out_s)
+    torch.cuda.synchronize()
+    words = (w.d + 31) // 32
+    assert torch.equal(out_s[:, :words], out[:, :words])
+    for c in sorted(set([0, 1, w.n // 2, w.n - 1])):
+        for hb in (0, 1):
+            sa, a = ctx.mailbox_tensor(c, hb)
+            sb, b = ctx_s.mailbox_tensor(c, hb)
+            assert sa == sb and torch.equal(a, b)
+    ctx.close()
+    ctx_s.close()
+    del H
+    torch.cuda.empty_cache()
+
+
+def test_full_size_sum_rule_cfg2():
+    """Plain ring-all-reduce at cfg2's size: fused and hop-by-hop give the same
+    float32 bits, sampled coordinates match the oracle's ring-order float32 sum."""
+    w = W.WORKLOADS["cfg2"]
+    H = W.honest_updates(w, 0, device="cuda")
+    outs = []
+    for mode in (B.AGG_FUSED, B.AGG_STEPWISE):
+        ctx = B.Brace(w.n, 0, w.d, B.default_params(rule=B.RULE_SUM, agg_mode=mode))
+        out = ctx.new_output()
+        ctx.aggregate(H, out)
+        torch.cuda.synchronize()
+        outs.append(out)
+        bounds = [ctx.segment(j) for j in range(w.n)]
+        ctx.close()
+    assert torch.equal(outs[0][:, :w.d].view(torch.int32), outs[1][:, :w.d].view(torch.int32))
+    for c in range(1, w.n):
+        assert torch.equal(outs[0][c, :w.d].view(torch.int32), outs[0][0, :w.d].view(torch.int32))
+    rng = np.random.default_rng(2)
+    idx = np.unique(np.concatenate([np.arange(0, 512), np.arange(w.d - 512, w.d), rng.integers(0, w.d, 4096)]))
+    Hs = H[:, torch.as_tensor(idx, device="cuda")].cpu().numpy()
+    got = outs[0][0, torch.as_tensor(idx, device="cuda")].cpu().numpy()
+    # sub-vector j is reduced starting at client j: same float32 add order, coordinate by coordinate
+    seg_of = np.searchsorted(np.array([b for b, _ in bounds] + [w.d]), idx, side="right") - 1
+    exp = np.empty(idx.size, dtype=np.float32)
+    for t, (k, j) in enumerate(zip(idx, seg_of)):
+        acc = Hs[j, t]
+        for i in range(1, w.n):
+            acc = np.float32(acc + Hs[(j + i) % w.n, t])
+        exp[t] = acc
+    assert np.array_equal(got.view(np.uint32), exp.view(np.uint32))
+    ref = O.sum_direct_f64(Hs)
+    scale = np.abs(Hs.astype(np.float64)).sum(0)
+    assert (np.abs(got.astype(np.float64) - ref) <= 1e-5 * np.maximum(np.abs(ref), scale)).all()
