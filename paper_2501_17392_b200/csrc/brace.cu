@@ -367,10 +367,30 @@ int inject_impl(brace_ctx* ctx, const brace_attack* atk, const float* H, int64_t
   if (kind == BRACE_ATTACK_SCALED_MEAN || kind == BRACE_ATTACK_MEAN_SHIFT) {
     const int m = ctx->n - ctx->f;
     const int mpad = (m + 7) / 8 * 8;
+    if (kind == BRACE_ATTACK_MEAN_SHIFT && m <= 127 && ctx->stats_vw == 0) {
+      // two passes: register-resident variant, one coordinate per thread, all honest values in registers
+      HonestRows rows;
+      for (int r = 0; r < 128; ++r)
+        rows.byte_off[r] = (int64_t)ctx->ids_on_device[(size_t)ctx->f + (size_t)(r < m ? r : m - 1)] * ld_h * 4;
+      const unsigned blocks = tiles(ctx->d, 128);
+#define BRACE_STATS_REG(MFULL)                                                                          \
+  case MFULL:                                                                                           \
+    inject_stats_reg_kernel<MFULL><<<blocks, 128, 0, st>>>(kind, rows, ctx->d_ids, ctx->f, m, H, Uo, ld_u, \
+                                                           ctx->d, atk->scale, atk->kappa);             \
+    break
+      switch (m / 8 * 8) {
+        BRACE_STATS_REG(0); BRACE_STATS_REG(8); BRACE_STATS_REG(16); BRACE_STATS_REG(24); BRACE_STATS_REG(32);
+        BRACE_STATS_REG(40); BRACE_STATS_REG(48); BRACE_STATS_REG(56); BRACE_STATS_REG(64); BRACE_STATS_REG(72);
+        BRACE_STATS_REG(80); BRACE_STATS_REG(88); BRACE_STATS_REG(96); BRACE_STATS_REG(104); BRACE_STATS_REG(112);
+        default: BRACE_STATS_REG(120);
+      }
+#undef BRACE_STATS_REG
+      return check_launch(ctx);
+    }
     // staged variant: one column (vw floats wide) of all m honest rows per thread in shared memory
     const bool rows8 = (ld_h % 2 == 0) && (ld_u % 2 == 0) && (reinterpret_cast<uintptr_t>(H) & 7u) == 0 &&
                        (reinterpret_cast<uintptr_t>(Uo) & 7u) == 0;
-    int vw = ctx->stats_vw > 0 ? ctx->stats_vw : 2;
+    int vw = ctx->stats_vw > 0 ? ctx->stats_vw : 4;
     if (vw == 4 && !rows16) vw = 2;
     if (vw == 2 && !rows8) vw = 1;
     const bool layout_ok = true;

@@ -741,4 +741,57 @@ __global__ void inject_stats_smem_kernel(int kind, const int* __restrict__ ids, 
   }
 }
 
+// Register-resident variant of the statistics kernel for up to 128 honest rows:
+// a thread owns one coordinate, requests all of its honest values at once (they
+// stay in registers), then runs the float64 sum and the float64 deviations over
+// them -- the second pass costs no memory traffic at all.  MFULL rows (a
+// multiple of 8) are handled without predicates, up to 7 more with.  Row byte
+// offsets travel as a kernel parameter so that, with the loops unrolled, every
+// row address is one 64-bit add with a constant operand.
+struct HonestRows {
+  int64_t byte_off[128];
+};
+
+template <int MFULL>
+__global__ void __launch_bounds__(128, (MFULL <= 24 ? 8 : (MFULL <= 40 ? 6 : (MFULL <= 56 ? 5 : (MFULL <= 80 ? 4 : (MFULL <= 96 ? 3 : 2))))))
+inject_stats_reg_kernel(int kind, const __grid_constant__ HonestRows rows, const int* __restrict__ ids, int f, int m,
+                        const float* H, float* Uo, int64_t ld_u, int64_t d, float scale, float kappa) {
+  constexpr int MTAIL = 7;
+  const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= d) return;
+  const char* src = reinterpret_cast<const char*>(H + k);
+  const int tail = m - MFULL;                        // 0..7 rows beyond the unpredicated ones
+  float x[MFULL + MTAIL];
+#pragma unroll
+  for (int r = 0; r < MFULL; ++r) x[r] = __ldcs(reinterpret_cast<const float*>(src + rows.byte_off[r]));
+#pragma unroll
+  for (int r = 0; r < MTAIL; ++r)
+    x[MFULL + r] = (r < tail) ? __ldcs(reinterpret_cast<const float*>(src + rows.byte_off[MFULL + r])) : 0.0f;
+  double tot = 0.0;
+#pragma unroll
+  for (int r = 0; r < MFULL; ++r) tot = __dadd_rn(tot, (double)x[r]);
+#pragma unroll
+  for (int r = 0; r < MTAIL; ++r)
+    if (r < tail) tot = __dadd_rn(tot, (double)x[MFULL + r]);
+  const double dm = (double)m;
+  const double mean = __ddiv_rn(tot, dm);
+  double vec;
+  if (kind == 3) {
+    vec = __dmul_rn((double)scale, mean);
+  } else {
+    double sq = 0.0;
+#pragma unroll
+    for (int r = 0; r < MFULL + MTAIL; ++r) {
+      if (r < MFULL || r - MFULL < tail) {
+        asm volatile("" : "+f"(x[r]));               // convert again rather than keep 2 registers per value
+        const double dev = __dsub_rn((double)x[r], mean);
+        sq = __dadd_rn(sq, __dmul_rn(dev, dev));
+      }
+    }
+    vec = __dsub_rn(mean, __dmul_rn((double)kappa, __dsqrt_rn(__ddiv_rn(sq, dm))));
+  }
+  const float v = __double2float_rn(vec);
+  for (int bq = 0; bq < f; ++bq) Uo[(int64_t)ids[bq] * ld_u + k] = v;
+}
+
 }  // namespace brace
