@@ -124,6 +124,23 @@ inline unsigned tiles(int64_t items, int64_t per_block) {
 
 // ---- launches of the per-hop kernels -------------------------------------------------
 
+// Launch with programmatic stream serialization: the kernel may begin while its
+// predecessor on the stream drains; it synchronises on the device (pdl_wait).
+template <typename... KArgs, typename... Args>
+void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 bool vec_layout_ok(const brace_ctx* ctx, const float* U, int64_t ld) {
   return (ctx->p.granule % 4 == 0) && (ld % 4 == 0) && aligned16(U);
 }
@@ -143,8 +160,8 @@ int launch_rs_step(brace_ctx* ctx, int step, const float* U, int64_t ld, cudaStr
   const bool zs = ctx->p.zero_sign != 0;
   const int zsv = ctx->p.zero_sign;
 #define BRACE_RS_SIGN(P, VPT, ZS)                                                                            \
-  rs_step_sign_kernel<P, VPT, ZS><<<grid, kThreads, 0, st>>>(ctx->pt, U, ld, (const P*)ctx->mail[in_set],    \
-                                                             (P*)ctx->mail[out_set], ctx->seg_pad, step, zsv)
+  launch_pdl(rs_step_sign_kernel<P, VPT, ZS>, grid, dim3(kThreads), st, ctx->pt, U, ld,                       \
+             (const P*)ctx->mail[in_set], (P*)ctx->mail[out_set], ctx->seg_pad, step, zsv)
 #define BRACE_RS_SIGN_P(P)                                                                         \
   do {                                                                                             \
     switch (vpt) {                                                                                 \
@@ -157,11 +174,11 @@ int launch_rs_step(brace_ctx* ctx, int step, const float* U, int64_t ld, cudaStr
   if (ctx->p.rule == BRACE_RULE_SUM) {
     dim3 gsum(tiles(ctx->seg_max, vec ? kThreads * 4 : kThreads), (unsigned)n);
     if (vec)
-      rs_step_sum_kernel<true><<<gsum, kThreads, 0, st>>>(ctx->pt, U, ld, (const float*)ctx->mail[in_set],
-                                                          (float*)ctx->mail[out_set], ctx->seg_pad, step);
+      launch_pdl(rs_step_sum_kernel<true>, gsum, dim3(kThreads), st, ctx->pt, U, ld,
+                 (const float*)ctx->mail[in_set], (float*)ctx->mail[out_set], ctx->seg_pad, step);
     else
-      rs_step_sum_kernel<false><<<gsum, kThreads, 0, st>>>(ctx->pt, U, ld, (const float*)ctx->mail[in_set],
-                                                           (float*)ctx->mail[out_set], ctx->seg_pad, step);
+      launch_pdl(rs_step_sum_kernel<false>, gsum, dim3(kThreads), st, ctx->pt, U, ld,
+                 (const float*)ctx->mail[in_set], (float*)ctx->mail[out_set], ctx->seg_pad, step);
   } else if (ctx->entry_bytes == 1) {
     BRACE_RS_SIGN_P(int8_t);
   } else {
@@ -179,19 +196,19 @@ int launch_consensus(brace_ctx* ctx, void* out, int64_t out_ld, cudaStream_t st)
     const bool vec = (ctx->p.granule % 4 == 0) && (out_ld % 4 == 0) && aligned16(out);
     dim3 grid(tiles(ctx->seg_max, vec ? kThreads * 4 : kThreads), (unsigned)n);
     if (vec)
-      consensus_sum_kernel<true><<<grid, kThreads, 0, st>>>(ctx->pt, (const float*)ctx->mail[set], ctx->seg_pad,
-                                                            (float*)out, out_ld, ctx->p.mean);
+      launch_pdl(consensus_sum_kernel<true>, grid, dim3(kThreads), st, ctx->pt, (const float*)ctx->mail[set],
+                 ctx->seg_pad, (float*)out, out_ld, ctx->p.mean);
     else
-      consensus_sum_kernel<false><<<grid, kThreads, 0, st>>>(ctx->pt, (const float*)ctx->mail[set], ctx->seg_pad,
-                                                             (float*)out, out_ld, ctx->p.mean);
+      launch_pdl(consensus_sum_kernel<false>, grid, dim3(kThreads), st, ctx->pt, (const float*)ctx->mail[set],
+                 ctx->seg_pad, (float*)out, out_ld, ctx->p.mean);
   } else {
     dim3 grid(tiles(ctx->seg_max / 32 + 2, kThreads), (unsigned)n);
     if (ctx->entry_bytes == 1)
-      consensus_sign_kernel<int8_t><<<grid, kThreads, 0, st>>>(ctx->pt, (const int8_t*)ctx->mail[set], ctx->seg_pad,
-                                                               (uint32_t*)out, out_ld, ctx->lam_i);
+      launch_pdl(consensus_sign_kernel<int8_t>, grid, dim3(kThreads), st, ctx->pt, (const int8_t*)ctx->mail[set],
+                 ctx->seg_pad, (uint32_t*)out, out_ld, ctx->lam_i);
     else
-      consensus_sign_kernel<int16_t><<<grid, kThreads, 0, st>>>(ctx->pt, (const int16_t*)ctx->mail[set],
-                                                                ctx->seg_pad, (uint32_t*)out, out_ld, ctx->lam_i);
+      launch_pdl(consensus_sign_kernel<int16_t>, grid, dim3(kThreads), st, ctx->pt, (const int16_t*)ctx->mail[set],
+                 ctx->seg_pad, (uint32_t*)out, out_ld, ctx->lam_i);
   }
   return check_launch(ctx);
 }
@@ -202,12 +219,12 @@ int launch_ag_step(brace_ctx* ctx, int step, void* out, int64_t out_ld, cudaStre
     const bool vec = (ctx->p.granule % 4 == 0) && (out_ld % 4 == 0) && aligned16(out);
     dim3 grid(tiles(ctx->seg_max, vec ? kThreads * 4 : kThreads), (unsigned)n);
     if (vec)
-      ag_step_f32_kernel<true><<<grid, kThreads, 0, st>>>(ctx->pt, (float*)out, out_ld, step);
+      launch_pdl(ag_step_f32_kernel<true>, grid, dim3(kThreads), st, ctx->pt, (float*)out, out_ld, step);
     else
-      ag_step_f32_kernel<false><<<grid, kThreads, 0, st>>>(ctx->pt, (float*)out, out_ld, step);
+      launch_pdl(ag_step_f32_kernel<false>, grid, dim3(kThreads), st, ctx->pt, (float*)out, out_ld, step);
   } else {
     dim3 grid(tiles(ctx->seg_max / 32 + 2, kThreads), (unsigned)n);
-    ag_step_bits_kernel<<<grid, kThreads, 0, st>>>(ctx->pt, (uint32_t*)out, out_ld, step);
+    launch_pdl(ag_step_bits_kernel, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, step);
   }
   return check_launch(ctx);
 }

@@ -35,6 +35,14 @@ __device__ __forceinline__ int sgn1(float x, int zs) {
   return s;
 }
 
+// Programmatic dependent launch: the per-hop kernels are launched so that the
+// next hop's CTAs may start while the current hop drains.  pdl_wait() returns
+// once every kernel launched before this one on the stream has completed and
+// its writes are visible; before it a kernel may only read memory that no
+// earlier kernel of the round writes (the update matrix, from hop 1 on).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // streaming (read-once) 128-bit load
 __device__ __forceinline__ float4 ld_stream(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
 
@@ -74,6 +82,8 @@ rs_step_sign_kernel(Part pt, const float* __restrict__ U, int64_t ld, const P* _
   const float* ur = U + (int64_t)r * ld + b;
   const P* in = mail_in + (int64_t)c * seg_pad;
   P* out = mail_out + (int64_t)r * seg_pad;
+  pdl_launch_dependents();
+  if (step == 0) pdl_wait();                      // whoever produced the updates must have finished
   if (VPT > 0) {
     constexpr int V = VPT > 0 ? VPT : 1;
     const int64_t base = (int64_t)blockIdx.x * (256 * V) + threadIdx.x;
@@ -82,13 +92,20 @@ rs_step_sign_kernel(Part pt, const float* __restrict__ U, int64_t ld, const P* _
     int a[V][4];
     bool full[V];
 #pragma unroll
-    for (int v = 0; v < V; ++v) {
+    for (int v = 0; v < V; ++v) {                  // own updates: independent of the previous hop
       const int64_t i = (base + v * 256) * 4;
       full[v] = i + 4 <= L;
       if (full[v]) {
         x[v] = ld_stream(ur + i);
         if (step == 0) y[v] = ld_stream(uc + i);
-        else load4(in + i, a[v][0], a[v][1], a[v][2], a[v][3]);
+      }
+    }
+    if (step != 0) {
+      pdl_wait();                                  // previous hop done: mailboxes readable, other set writable
+#pragma unroll
+      for (int v = 0; v < V; ++v) {
+        const int64_t i = (base + v * 256) * 4;
+        if (full[v]) load4(in + i, a[v][0], a[v][1], a[v][2], a[v][3]);
       }
     }
 #pragma unroll
@@ -109,6 +126,7 @@ rs_step_sign_kernel(Part pt, const float* __restrict__ U, int64_t ld, const P* _
       }
     }
   } else {
+    if (step != 0) pdl_wait();
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t < L) {
       int s0 = (step == 0) ? sgn1<ZS>(uc[t], zs) : (int)in[t];
@@ -134,18 +152,23 @@ rs_step_sum_kernel(Part pt, const float* __restrict__ U, int64_t ld, const float
   const float* in = (step == 0) ? uc : mail_in + (int64_t)c * seg_pad;
   float* out = mail_out + (int64_t)r * seg_pad;
   const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  pdl_launch_dependents();
+  if (step == 0) pdl_wait();
   if (VEC) {
     const int64_t i = t * 4;
     if (i + 4 <= L) {
       float4 x = ld_stream(ur + i);
+      if (step != 0) pdl_wait();
       float4 y = (step == 0) ? ld_stream(in + i) : *reinterpret_cast<const float4*>(in + i);
       float4 o;
       o.x = __fadd_rn(y.x, x.x); o.y = __fadd_rn(y.y, x.y); o.z = __fadd_rn(y.z, x.z); o.w = __fadd_rn(y.w, x.w);
       *reinterpret_cast<float4*>(out + i) = o;
     } else {
+      if (step != 0) pdl_wait();
       for (int64_t k = i; k < L; ++k) out[k] = __fadd_rn(in[k], ur[k]);
     }
   } else {
+    if (step != 0) pdl_wait();
     if (t < L) out[t] = __fadd_rn(in[t], ur[t]);
   }
 }
@@ -159,6 +182,8 @@ template <typename P>
 __global__ void __launch_bounds__(256)
 consensus_sign_kernel(Part pt, const P* __restrict__ mail, int64_t seg_pad, uint32_t* __restrict__ out,
                       int64_t out_ld, int lam) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int n = pt.n;
   const int c = blockIdx.y;
   const int j = next_client(c, n);
@@ -195,6 +220,8 @@ template <bool VEC>
 __global__ void __launch_bounds__(256)
 consensus_sum_kernel(Part pt, const float* __restrict__ mail, int64_t seg_pad, float* __restrict__ out,
                      int64_t out_ld, int mean) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int n = pt.n;
   const int c = blockIdx.y;
   const int j = next_client(c, n);
@@ -223,6 +250,8 @@ consensus_sum_kernel(Part pt, const float* __restrict__ mail, int64_t seg_pad, f
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 ag_step_bits_kernel(Part pt, uint32_t* out, int64_t out_ld, int step) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int n = pt.n;
   const int c = blockIdx.y;
   const int r = next_client(c, n);
@@ -248,6 +277,8 @@ ag_step_bits_kernel(Part pt, uint32_t* out, int64_t out_ld, int step) {
 template <bool VEC>
 __global__ void __launch_bounds__(256)
 ag_step_f32_kernel(Part pt, float* out, int64_t out_ld, int step) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int n = pt.n;
   const int c = blockIdx.y;
   const int r = next_client(c, n);
