@@ -217,7 +217,7 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
  * prefetched) in {(1,8),(2,4),(1,4),(2,8),(1,16)}; fused_grid = 0 launches one
  * CTA per tile, > 0 caps the grid (CTAs then loop over tiles).  Adding 10, 20
  * or 40 to fused_variant makes the share-reduce hop kernel process 1, 2 or 4
- * float4 per thread (default: 2, fewer for short sub-vectors).  Results do not
+ * float4 per thread (default: 4, fewer for short sub-vectors).  Results do not
  * depend on any of these. */
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid);
 

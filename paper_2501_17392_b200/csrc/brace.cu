@@ -152,7 +152,7 @@ int launch_rs_step(brace_ctx* ctx, int step, const float* U, int64_t ld, cudaStr
   // float4 per thread: enough loads in flight for long sub-vectors, enough CTAs for short ones
   int vpt = 0;
   if (vec) {
-    vpt = ctx->step_vpt > 0 ? ctx->step_vpt : 2;
+    vpt = ctx->step_vpt > 0 ? ctx->step_vpt : 4;
     while (vpt > 1 && (int64_t)n * ((ctx->seg_max + 1024 * vpt - 1) / (1024 * vpt)) < 4 * kSmCount) vpt >>= 1;
   }
   const int64_t per_block = vec ? (int64_t)kThreads * 4 * vpt : kThreads;
@@ -223,8 +223,14 @@ int launch_ag_step(brace_ctx* ctx, int step, void* out, int64_t out_ld, cudaStre
     else
       launch_pdl(ag_step_f32_kernel<false>, grid, dim3(kThreads), st, ctx->pt, (float*)out, out_ld, step);
   } else {
-    dim3 grid(tiles(ctx->seg_max / 32 + 2, kThreads), (unsigned)n);
-    launch_pdl(ag_step_bits_kernel, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, step);
+    const bool wide = (ctx->p.granule % 128 == 0) && (out_ld % 4 == 0) && aligned16(out);
+    if (wide) {
+      dim3 grid(tiles(ctx->seg_max / 128 + 2, kThreads), (unsigned)n);
+      launch_pdl(ag_step_bits_kernel<4>, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, step);
+    } else {
+      dim3 grid(tiles(ctx->seg_max / 32 + 2, kThreads), (unsigned)n);
+      launch_pdl(ag_step_bits_kernel<1>, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, step);
+    }
   }
   return check_launch(ctx);
 }

@@ -248,6 +248,9 @@ consensus_sum_kernel(Part pt, const float* __restrict__ mail, int64_t seg_pad, f
 // ---------------------------------------------------------------------------
 // Share-Only hop (Section 3 Phase IV): row c -> row (c+1) mod n, one sub-vector.
 // ---------------------------------------------------------------------------
+// WPT = words per thread: 4 copies 128 bits at a time (needs 16-byte aligned rows
+// and granule % 128 == 0); boundary words of a sub-vector are always masked.
+template <int WPT>
 __global__ void __launch_bounds__(256)
 ag_step_bits_kernel(Part pt, uint32_t* out, int64_t out_ld, int step) {
   pdl_launch_dependents();
@@ -261,17 +264,27 @@ ag_step_bits_kernel(Part pt, uint32_t* out, int64_t out_ld, int step) {
   const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
   if (b >= e) return;
   const int64_t w0 = b >> 5, w1 = (e + 31) >> 5;
-  const int64_t w = w0 + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (w >= w1) return;
-  const int64_t k0 = (w << 5) > b ? (w << 5) : b;
-  const int64_t k1 = ((w + 1) << 5) < e ? ((w + 1) << 5) : e;
-  const int lo = (int)(k0 & 31);
-  int hi = (int)(k1 - (w << 5));
-  if (k1 == pt.d) hi = 32;
-  const uint32_t mask = (hi == 32 ? 0xffffffffu : ((1u << hi) - 1u)) & ~((1u << lo) - 1u);
-  const uint32_t v = out[(int64_t)c * out_ld + w];
-  uint32_t* dst = out + (int64_t)r * out_ld + w;
-  *dst = (mask == 0xffffffffu) ? v : ((*dst & ~mask) | (v & mask));
+  const int64_t wt = w0 + ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * WPT;
+  if (wt >= w1) return;
+  const uint32_t* src = out + (int64_t)c * out_ld;
+  uint32_t* dst = out + (int64_t)r * out_ld;
+  if (WPT == 4 && (wt << 5) >= b && ((wt + 4) << 5) <= e) {      // four whole words inside the sub-vector
+    *reinterpret_cast<uint4*>(dst + wt) = *reinterpret_cast<const uint4*>(src + wt);
+    return;
+  }
+#pragma unroll
+  for (int q = 0; q < WPT; ++q) {
+    const int64_t w = wt + q;
+    if (w >= w1) break;
+    const int64_t k0 = (w << 5) > b ? (w << 5) : b;
+    const int64_t k1 = ((w + 1) << 5) < e ? ((w + 1) << 5) : e;
+    const int lo = (int)(k0 & 31);
+    int hi = (int)(k1 - (w << 5));
+    if (k1 == pt.d) hi = 32;
+    const uint32_t mask = (hi == 32 ? 0xffffffffu : ((1u << hi) - 1u)) & ~((1u << lo) - 1u);
+    const uint32_t v = src[w];
+    dst[w] = (mask == 0xffffffffu) ? v : ((dst[w] & ~mask) | (v & mask));
+  }
 }
 
 template <bool VEC>
