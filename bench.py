@@ -324,20 +324,30 @@ def run_cuda(args, w):
     entry_bytes = 1 if n <= 127 else 2
     fused_used = (args.mode != "stepwise")
     agg_avg_ms = float(np.mean(agg_ms))
+    inj_avg_ms = float(np.mean(inj_ms))
+    words = (d + 31) // 32
     if fused_used:
-        alg = algorithmic_bytes_fused(n, d, entry_bytes)
-        kernel_name = "fused_sign_kernel"
+        agg_alg = algorithmic_bytes_fused(n, d, entry_bytes)
+        agg_kernel = "fused_sign_kernel"
         launches_per_step = 2
     else:
-        words = (d + 31) // 32
-        alg = 4 * n * d + (n - 2) * d + (n - 1) * d + d + 4 * words + (n - 1) * 2 * 4 * words
-        kernel_name = "rs_step_sign_kernel (+consensus, share-only hops)"
+        agg_alg = 4 * n * d + (n - 2) * d + (n - 1) * d + d + 4 * words + (n - 1) * 2 * 4 * words
+        agg_kernel = "rs_step_sign_kernel x(n-1) + consensus_sign_kernel + ag_step_bits_kernel x(n-1)"
         launches_per_step = 1 + 2 * (n - 1) + 1
-    achieved = alg / (agg_avg_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+    inj_alg, inj_kernel = injection_bytes(w)
+
+    def roof(kernel, alg, ms, traffic_key):
+        achieved = alg / (ms * 1e-3) / 1e9
+        return {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"{peak_kind} device copy",
-                "algorithmic_bytes_per_launch": alg, "ms_per_launch": agg_avg_ms,
-                "traffic": TRAFFIC_BYTES.get(w.name)}
+                "algorithmic_bytes_per_launch": alg, "ms_per_launch": ms,
+                "traffic": TRAFFIC_BYTES.get((w.name, traffic_key)) if not args.d else None}
+
+    roof_agg = roof(agg_kernel, agg_alg, agg_avg_ms, "aggregate")
+    roof_inj = roof(inj_kernel, inj_alg, inj_avg_ms, "inject")
+    # the roofline entry is the kernel that takes the larger share of the step
+    roofline = roof_inj if inj_avg_ms > agg_avg_ms else roof_agg
+    roofline["other_kernel"] = roof_agg if roofline is roof_inj else roof_inj
 
     cpu_baseline = None
     if not args.no_cpu:
@@ -358,7 +368,7 @@ def run_cuda(args, w):
                    "replicas": world, "parallelism": "replicas only"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline, "cpu_baseline": cpu_baseline,
-        "phases_ms": {"inject": float(np.mean(inj_ms)), "aggregate": agg_avg_ms},
+        "phases_ms": {"inject": inj_avg_ms, "aggregate": agg_avg_ms},
         "aggregate_only_elements_per_s": n * d / (agg_avg_ms * 1e-3),
         "stepwise": stepwise,
     }
@@ -368,9 +378,26 @@ def run_cuda(args, w):
         dist.destroy_process_group()
 
 
-# DRAM bytes per launch of the fused kernel from an ncu capture (profiles/), by workload;
-# None where no capture of the current kernel exists.
-TRAFFIC_BYTES: dict = {}
+def injection_bytes(w):
+    """(algorithmic bytes, kernel name) of one injection launch."""
+    n, f, d = w.n, w.f, w.d
+    if w.attack == W.ATTACK_SCALE_OWN:
+        return 8 * f * d, "inject_elementwise_vec_kernel"
+    if w.attack == W.ATTACK_GAUSSIAN:
+        return 8 * f * d, "inject_elementwise_vec_kernel"
+    if w.attack == W.ATTACK_SPARSE_NOISE:
+        return 12 * f * d, "inject_elementwise_vec_kernel"
+    if w.attack == W.ATTACK_SCALED_MEAN:
+        return 4 * (n - f) * d + 4 * f * d, "inject_stats_smem_kernel"
+    return 4 * (n - f) * d + 4 * f * d, "inject_stats_reg_kernel"
+
+
+# DRAM bytes (read + write) per launch from ncu captures of the full-size workload
+# (profiles/), keyed by (workload, phase); absent where no capture of the current kernel exists.
+TRAFFIC_BYTES: dict = {
+    ("cfg4", "aggregate"): 10_223_567_000 + 328_103_000,   # fused_sign_kernel<int8,1,8>, profiles/fused_sign_kernel_cfg4.md
+    ("cfg4", "inject"): 8_178_284_000 + 1_985_047_000,     # inject_stats_reg_kernel<80>, profiles/inject_stats_reg_kernel_cfg4.md
+}
 
 
 def main():
