@@ -41,17 +41,28 @@ typedef void* brace_stream_t; /* cudaStream_t */
 enum {
   BRACE_OK = 0,
   BRACE_ERR_INVALID_ARG = 1, /* null / out-of-range / misaligned argument; nothing was launched */
-  BRACE_ERR_UNSUPPORTED = 2, /* valid request this build cannot serve (e.g. n > 32767)          */
+  BRACE_ERR_UNSUPPORTED = 2, /* valid request the library cannot serve (e.g. n > 32767)         */
   BRACE_ERR_BAD_STEP = 3,    /* hop called out of order; nothing was launched                   */
   BRACE_ERR_WORKSPACE = 4,   /* workspace missing, too small or misaligned                      */
   BRACE_ERR_CUDA = 5,        /* a CUDA runtime call failed; see brace_last_cuda_error           */
   BRACE_ERR_TIMEOUT = 6      /* reserved: a bounded device-side wait ran out                    */
 };
 
-/* aggregation rules */
+/* aggregation rules.  All but SUM share Phases I, II and IV of Section 3 (sign,
+ * share-reduce of the signs, 1-bit share-only) and differ in the Phase III map
+ * applied to the integer sign-sum S = sum_i sign(g_i[k]):
+ *   SIGN_CONSENSUS  +1 if S > lambda, else -1                       (BRACE, Eq. (1))
+ *   MAJORITY_SIGN   +1 if S > 0, else -1 (lambda unused)            (signSGD with majority vote run over the
+ *                   ring, which Section 5.2 says follows the same procedure; the paper does not say what a tie
+ *                   S = 0 gives: here -1, as Eq. (1) does with lambda = 0)
+ *   ABS_CONSENSUS   +1 if |S| > lambda, else -1                     (the RLR-style test Section 5.2 describes:
+ *                   the absolute value of the sum, positive and negative agreement treated alike; the paper
+ *                   gives no formula, strictness of the inequality follows Eq. (1))                          */
 enum {
   BRACE_RULE_SIGN_CONSENSUS = 0, /* BRACE, Section 3, Eq. (1)                                     */
-  BRACE_RULE_SUM = 1             /* plain ring-all-reduce sum, Section 2.2 (optionally the mean)  */
+  BRACE_RULE_SUM = 1,            /* plain ring-all-reduce sum, Section 2.2 (optionally the mean)  */
+  BRACE_RULE_MAJORITY_SIGN = 2,  /* sign of the sign-sum (Section 5.2: signSGD over the ring)     */
+  BRACE_RULE_ABS_CONSENSUS = 3   /* |sign-sum| against lambda (Section 5.2: RLR over the ring)    */
 };
 
 /* how brace_aggregate runs a round (the result is the same) */

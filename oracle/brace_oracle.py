@@ -42,6 +42,9 @@ import numpy as np
 
 RULE_SIGN_CONSENSUS = 0  # BRACE, Section 3, Eq. (1)
 RULE_SUM = 1             # plain ring-all-reduce, Section 2.2
+RULE_MAJORITY_SIGN = 2   # signSGD with majority vote over the ring (Section 5.2)
+RULE_ABS_CONSENSUS = 3   # RLR-style test on |sign-sum| over the ring (Section 5.2)
+SIGN_RULES = (RULE_SIGN_CONSENSUS, RULE_MAJORITY_SIGN, RULE_ABS_CONSENSUS)
 
 ATTACK_SCALE_OWN = 1     # b_i = a * h_i
 ATTACK_GAUSSIAN = 2      # b_i = sigma * z_i
@@ -95,10 +98,33 @@ def lambda_int(lam: float, n: int) -> int:
 
 
 # --------------------------------------------------------------------------
+# Section 3, Phase III: the map applied to the integer sign-sum S
+# --------------------------------------------------------------------------
+def consensus_map(total: np.ndarray, rule: int, lam: float, n: int) -> np.ndarray:
+    """+-1 vector from the sign-sums.
+
+    RULE_SIGN_CONSENSUS  Eq. (1): +1 if S > lambda else -1.
+    RULE_MAJORITY_SIGN   Section 5.2, signSGD carried over the ring: the sign of
+                         S; the paper does not say what S = 0 gives, here -1.
+    RULE_ABS_CONSENSUS   Section 5.2, the RLR-style test: "the absolute value of
+                         the sum", positive and negative agreement alike:
+                         +1 if |S| > lambda else -1 (strictness as in Eq. (1)).
+    """
+    if rule == RULE_SIGN_CONSENSUS:
+        return np.where(total > lambda_int(lam, n), 1, -1).astype(np.int8)
+    if rule == RULE_MAJORITY_SIGN:
+        return np.where(total > 0, 1, -1).astype(np.int8)
+    if rule == RULE_ABS_CONSENSUS:
+        return np.where(np.abs(total) > lambda_int(lam, n), 1, -1).astype(np.int8)
+    raise ValueError("not a sign rule")
+
+
+# --------------------------------------------------------------------------
 # Section 3, Phase III, Eq. (1): the aggregation rule as a plain definition
 # --------------------------------------------------------------------------
-def gar_direct(updates: np.ndarray, lam: float, zero_sign: int = 0) -> np.ndarray:
-    """GAR(g_1..g_n)[k] = +1 if sum_i sign(g_i[k]) > lambda else -1 (Eq. (1)).
+def gar_direct(updates: np.ndarray, lam: float, zero_sign: int = 0, rule: int = RULE_SIGN_CONSENSUS) -> np.ndarray:
+    """GAR(g_1..g_n)[k] = +1 if sum_i sign(g_i[k]) > lambda else -1 (Eq. (1));
+    other sign rules swap the final map, see ``consensus_map``.
 
     updates: [n, d].  Returns int8 [d] with entries in {-1, +1}.
     """
@@ -107,8 +133,7 @@ def gar_direct(updates: np.ndarray, lam: float, zero_sign: int = 0) -> np.ndarra
     total = np.zeros(updates.shape[1], dtype=np.int32)
     for i in range(n):
         total = total + sgn(updates[i], zero_sign)
-    lam_i = lambda_int(lam, n)
-    return np.where(total > lam_i, 1, -1).astype(np.int8)
+    return consensus_map(total, rule, lam, n)
 
 
 def sign_sum_direct(updates: np.ndarray, zero_sign: int = 0) -> np.ndarray:
@@ -197,7 +222,7 @@ def ring_round(updates: np.ndarray, rule: int = RULE_SIGN_CONSENSUS, lam: float 
     bounds = partition(n, d, granule)
 
     # Phase I (BRACE) / local copies (SUM): one full-length working vector per client
-    if rule == RULE_SIGN_CONSENSUS:
+    if rule in SIGN_RULES:
         work = [sgn(updates[c], zero_sign) for c in range(n)]
     elif rule == RULE_SUM:
         work = [np.array(updates[c], dtype=np.float32, copy=True) for c in range(n)]
@@ -235,13 +260,12 @@ def ring_round(updates: np.ndarray, rule: int = RULE_SIGN_CONSENSUS, lam: float 
         trace.owned.append((j, work[c][b:e].copy()))
 
     # Phase III: Consensus (BRACE) / identity or mean (SUM), local to the owner
-    if rule == RULE_SIGN_CONSENSUS:
-        lam_i = lambda_int(lam, n)
+    if rule in SIGN_RULES:
         result = [np.zeros(d, dtype=np.int8) for _ in range(n)]
         for c in range(n):
             j = (c + 1) % n
             b, e = bounds[j]
-            result[c][b:e] = np.where(work[c][b:e] > lam_i, 1, -1).astype(np.int8)
+            result[c][b:e] = consensus_map(work[c][b:e], rule, lam, n)
     else:
         result = [np.zeros(d, dtype=np.float32) for _ in range(n)]
         for c in range(n):
@@ -286,7 +310,7 @@ def sum_direct_f64(updates: np.ndarray) -> np.ndarray:
 def sent_bits(trace: RingTrace, m_bits: int, rule: int) -> np.ndarray:
     """Bits sent per client: share-reduce moves m bits per coordinate; share-only
     moves 1 bit per coordinate under BRACE and m bits under plain RAR."""
-    ag_width = 1 if rule == RULE_SIGN_CONSENSUS else m_bits
+    ag_width = 1 if rule in SIGN_RULES else m_bits
     return trace.rs_sent * m_bits + trace.ag_sent * ag_width
 
 

@@ -16,7 +16,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libbrace.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BAD_STEP, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
-RULE_SIGN_CONSENSUS, RULE_SUM = 0, 1
+RULE_SIGN_CONSENSUS, RULE_SUM, RULE_MAJORITY_SIGN, RULE_ABS_CONSENSUS = 0, 1, 2, 3
 AGG_AUTO, AGG_STEPWISE, AGG_FUSED = 0, 1, 2
 ATTACK_NONE, ATTACK_SCALE_OWN, ATTACK_GAUSSIAN, ATTACK_SCALED_MEAN, ATTACK_MEAN_SHIFT, ATTACK_SPARSE_NOISE = range(6)
 

@@ -34,6 +34,7 @@ struct brace_ctx {
   brace_params p{};
   Part pt{};
   int lam_i = 0;
+  int lam_lo = 0;
   int entry_bytes = 1;
   int64_t seg_max = 0, seg_pad = 0;
   char* ws = nullptr;
@@ -59,7 +60,7 @@ namespace {
 
 bool params_ok(const brace_params* p) {
   if (!p) return false;
-  if (p->rule != BRACE_RULE_SIGN_CONSENSUS && p->rule != BRACE_RULE_SUM) return false;
+  if (p->rule < BRACE_RULE_SIGN_CONSENSUS || p->rule > BRACE_RULE_ABS_CONSENSUS) return false;
   if (!std::isfinite(p->lambda)) return false;
   if (p->zero_sign < -1 || p->zero_sign > 1) return false;
   if (p->granule < 1) return false;
@@ -104,6 +105,25 @@ size_t workspace_need(int n, int64_t d, const brace_params* p) {
   const int64_t pad = round_up(longest > 0 ? longest : 1, kMailAlign);
   const size_t one_set = (size_t)round_up((int64_t)n * pad * eb, 256);
   return 2 * one_set + ids_bytes(n);
+}
+
+// Integer thresholds of the consensus map bit = (S > hi) | (S < lo), S in [-n, n].
+void consensus_thresholds(const brace_params* p, int n, int* hi, int* lo) {
+  double fl = std::floor((double)p->lambda);
+  if (fl < -(double)n - 1.0) fl = -(double)n - 1.0;
+  if (fl > (double)n) fl = (double)n;
+  const int never = -2147483647 - 1;
+  if (p->rule == BRACE_RULE_MAJORITY_SIGN) {         // sign of the sign-sum; a tie gives -1
+    *hi = 0;
+    *lo = never;
+  } else if (p->rule == BRACE_RULE_ABS_CONSENSUS) {  // |S| > lambda, both directions count alike
+    *hi = (int)fl;
+    *lo = -(int)fl;
+    if (fl < 0.0) { *hi = -n - 1; *lo = never; }     // |S| >= 0 > lambda: always +1
+  } else {                                           // Eq. (1)
+    *hi = (int)fl;
+    *lo = never;
+  }
 }
 
 int cuda_fail(brace_ctx* ctx, cudaError_t err) {
@@ -205,10 +225,10 @@ int launch_consensus(brace_ctx* ctx, void* out, int64_t out_ld, cudaStream_t st)
     dim3 grid(tiles(ctx->seg_max / 32 + 2, kThreads), (unsigned)n);
     if (ctx->entry_bytes == 1)
       launch_pdl(consensus_sign_kernel<int8_t>, grid, dim3(kThreads), st, ctx->pt, (const int8_t*)ctx->mail[set],
-                 ctx->seg_pad, (uint32_t*)out, out_ld, ctx->lam_i);
+                 ctx->seg_pad, (uint32_t*)out, out_ld, ctx->lam_i, ctx->lam_lo);
     else
       launch_pdl(consensus_sign_kernel<int16_t>, grid, dim3(kThreads), st, ctx->pt, (const int16_t*)ctx->mail[set],
-                 ctx->seg_pad, (uint32_t*)out, out_ld, ctx->lam_i);
+                 ctx->seg_pad, (uint32_t*)out, out_ld, ctx->lam_i, ctx->lam_lo);
   }
   return check_launch(ctx);
 }
@@ -262,6 +282,7 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
   a.out = out;
   a.out_ld = out_ld;
   a.lam = ctx->lam_i;
+  a.lam_lo = ctx->lam_lo;
   a.zs = ctx->p.zero_sign;
   a.mean = ctx->p.mean;
   const bool zs = ctx->p.zero_sign != 0;
@@ -570,10 +591,7 @@ int brace_init(brace_ctx** out, int32_t n, int32_t f, int64_t d, const brace_par
   ctx->d = d;
   ctx->p = *params;
   ctx->pt = make_part(n, d, params->granule);
-  double fl = std::floor((double)params->lambda);
-  if (fl < -(double)n - 1.0) fl = -(double)n - 1.0;
-  if (fl > (double)n) fl = (double)n;
-  ctx->lam_i = (int)fl;
+  consensus_thresholds(params, n, &ctx->lam_i, &ctx->lam_lo);
   ctx->entry_bytes = eb;
   ctx->seg_max = longest_segment(ctx->pt);
   ctx->seg_pad = round_up(ctx->seg_max > 0 ? ctx->seg_max : 1, kMailAlign);
@@ -784,10 +802,7 @@ int brace_aggregate_static(int32_t n, int64_t d, const brace_params* params, con
   ctx.d = d;
   ctx.p = *params;
   ctx.pt = pt;
-  double fl = std::floor((double)params->lambda);
-  if (fl < -(double)n - 1.0) fl = -(double)n - 1.0;
-  if (fl > (double)n) fl = (double)n;
-  ctx.lam_i = (int)fl;
+  consensus_thresholds(params, n, &ctx.lam_i, &ctx.lam_lo);
   ctx.entry_bytes = eb;
   ctx.seg_max = seg_max;
   ctx.seg_pad = seg_pad;

@@ -175,13 +175,15 @@ rs_step_sum_kernel(Part pt, const float* __restrict__ U, int64_t ld, const float
 
 // ---------------------------------------------------------------------------
 // Consensus, Eq. (1): one thread per 32-bit output word of the owner's sub-vector.
+// The map is bit = (S > lam) | (S < lam_lo): Eq. (1) uses lam_lo = INT_MIN (never
+// true); the symmetric |S| > theta variant uses lam = theta, lam_lo = -theta.
 // Words that straddle a sub-vector boundary (granule % 32 != 0) are
 // read-modify-written; in one launch each row is written by one sub-vector only.
 // ---------------------------------------------------------------------------
 template <typename P>
 __global__ void __launch_bounds__(256)
 consensus_sign_kernel(Part pt, const P* __restrict__ mail, int64_t seg_pad, uint32_t* __restrict__ out,
-                      int64_t out_ld, int lam) {
+                      int64_t out_ld, int lam, int lam_lo) {
   pdl_launch_dependents();
   pdl_wait();
   const int n = pt.n;
@@ -203,9 +205,9 @@ consensus_sign_kernel(Part pt, const P* __restrict__ mail, int64_t seg_pad, uint
     for (int q = 0; q < NV; ++q) raw[q] = reinterpret_cast<const uint4*>(src + (k0 - b))[q];
     const P* v = reinterpret_cast<const P*>(raw);
 #pragma unroll
-    for (int q = 0; q < 32; ++q) bits |= (uint32_t)((int)v[q] > lam) << q;
+    for (int q = 0; q < 32; ++q) bits |= (uint32_t)(((int)v[q] > lam) | ((int)v[q] < lam_lo)) << q;
   } else {
-    for (int64_t k = k0; k < k1; ++k) bits |= (uint32_t)((int)src[k - b] > lam) << (int)(k & 31);
+    for (int64_t k = k0; k < k1; ++k) bits |= (uint32_t)(((int)src[k - b] > lam) | ((int)src[k - b] < lam_lo)) << (int)(k & 31);
   }
   const int lo = (int)(k0 & 31);
   int hi = (int)(k1 - (w << 5));                    // one past the last bit this sub-vector owns
@@ -335,7 +337,8 @@ struct FusedArgs {
   int64_t seg_pad;
   void* out;
   int64_t out_ld;
-  int lam;
+  int lam;      // consensus bit = (S > lam) | (S < lam_lo)
+  int lam_lo;
   int zs;
   int mean;
   int tiles_per_seg;
@@ -422,7 +425,7 @@ fused_sign_kernel(const FusedArgs a) {
     for (int v = 0; v < VPT; ++v) {
       uint32_t nib = 0;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) nib |= (uint32_t)(q < nv[v] && acc[v][q] > a.lam) << q;
+      for (int q = 0; q < 4; ++q) nib |= (uint32_t)(q < nv[v] && ((acc[v][q] > a.lam) | (acc[v][q] < a.lam_lo))) << q;
       uint32_t word = nib << (4 * (lane & 7));
       word |= __shfl_xor_sync(0xffffffffu, word, 1);
       word |= __shfl_xor_sync(0xffffffffu, word, 2);

@@ -210,6 +210,29 @@ def test_hop_by_hop_and_whole_round(n, d, G, ld, lam, zs, rule):
     ctx.close()
 
 
+@pytest.mark.parametrize("rule", [B.RULE_MAJORITY_SIGN, B.RULE_ABS_CONSENSUS])
+@pytest.mark.parametrize("n,d,G,ld,lam", [(8, 100_000, 128, 100_096, 2.0), (5, 4_099, 128, 4_100, 1.5),
+                                          (7, 12_345, 4, 12_348, 0.0), (20, 70_001, 128, 70_004, -1.0),
+                                          (3, 1_000, 32, 1_000, 1.0), (128, 9_000, 128, 9_088, 30.0)])
+def test_other_sign_rules(rule, n, d, G, ld, lam):
+    """Majority sign and |S| > lambda on the same schedule: only the Phase III map differs."""
+    U = W.small_integer_updates(n, d, seed=n * d, ld=ld, lo=-2, hi=2)
+    Uh = U.numpy()[:, :d]
+    tr = O.ring_round(Uh, rule=rule, lam=lam, granule=G)
+    assert np.array_equal(tr.outputs[0], O.gar_direct(Uh, lam, rule=rule))
+    Ud = U.cuda()
+    ctx = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, granule=G, agg_mode=B.AGG_STEPWISE))
+    out = ctx.new_output()
+    run_steps_and_check(ctx, Ud, tr, out, rule, d)
+    check_final(out, tr, rule, d)
+    ctx.close()
+    ctxa = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, granule=G))      # fused when the layout allows
+    out2 = torch.full_like(out, 3)
+    ctxa.aggregate(Ud, out2)
+    check_final(out2, tr, rule, d)
+    ctxa.close()
+
+
 def test_unaligned_rows_fall_back_to_scalar_kernels():
     """Row stride not a multiple of 4 and a base pointer off 16 bytes."""
     n, d, ld = 6, 3_001, 3_003

@@ -373,3 +373,47 @@ def test_inject_under_brace_sign_flip_equivalence():
     b = H.copy()
     b[0] = -H[0]
     assert np.array_equal(O.gar_direct(a, 0), O.gar_direct(b, 0))
+
+
+# ---------------------------------------------------------------- the other sign rules of Section 5.2
+@pytest.mark.parametrize("n", [2, 3, 4, 5])
+def test_majority_sign_and_abs_consensus_brute_force(n):
+    """All 3^n patterns; expected values from counting digits with Python integers:
+    majority sign = +1 iff positives outnumber negatives (tie -> -1);
+    abs consensus = +1 iff |positives - negatives| > lambda."""
+    patterns = list(itertools.product([0, 1, 2], repeat=n))
+    d = len(patterns)
+    U = np.zeros((n, d), dtype=np.float32)
+    for k, pat in enumerate(patterns):
+        for i, t in enumerate(pat):
+            U[i, k] = (t - 1) * (0.25 + i)
+    margin = [sum(1 for t in p if t == 2) - sum(1 for t in p if t == 0) for p in patterns]
+    for G in (1, 4, 128):
+        tr = O.ring_round(U, rule=O.RULE_MAJORITY_SIGN, lam=3.0, granule=G, keep_states=False)   # lambda is ignored
+        assert tr.outputs[0].tolist() == [1 if m > 0 else -1 for m in margin]
+        assert (tr.outputs == tr.outputs[0]).all()
+        for lam in range(-2, n + 1):
+            tr = O.ring_round(U, rule=O.RULE_ABS_CONSENSUS, lam=lam, granule=G, keep_states=False)
+            assert tr.outputs[0].tolist() == [1 if abs(m) > lam else -1 for m in margin]
+            assert (tr.outputs == tr.outputs[0]).all()
+            assert np.array_equal(O.gar_direct(U, lam, rule=O.RULE_ABS_CONSENSUS), tr.outputs[0])
+    assert np.array_equal(O.gar_direct(U, 0, rule=O.RULE_MAJORITY_SIGN), O.gar_direct(U, 0))   # == Eq. (1), lambda 0
+
+
+def test_abs_consensus_is_symmetric_and_is_the_union_of_both_directions():
+    rng = np.random.default_rng(21)
+    n, d = 11, 4000
+    U = rng.standard_normal((n, d)).astype(np.float32)
+    U[rng.random((n, d)) < 0.2] = 0
+    for lam in (0, 2, 4.5, 10):
+        a = O.gar_direct(U, lam, rule=O.RULE_ABS_CONSENSUS)
+        assert np.array_equal(a, O.gar_direct(-U, lam, rule=O.RULE_ABS_CONSENSUS))
+        both = np.maximum(O.gar_direct(U, lam), O.gar_direct(-U, lam))
+        assert np.array_equal(a, both)
+    assert (O.gar_direct(U, -1, rule=O.RULE_ABS_CONSENSUS) == 1).all()
+    assert (O.gar_direct(U, n, rule=O.RULE_ABS_CONSENSUS) == -1).all()
+    # sent bits equal BRACE's (Section 5.2: same communication cost)
+    V = rng.standard_normal((4, 8)).astype(np.float32)
+    for rule in (O.RULE_MAJORITY_SIGN, O.RULE_ABS_CONSENSUS):
+        tr = O.ring_round(V, rule=rule, lam=1, granule=1, keep_states=False)
+        assert O.sent_bits(tr, 8, rule).tolist() == [54] * 4      # Table 1 row n=4, d=8, m=8
