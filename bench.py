@@ -318,6 +318,42 @@ def run_cuda(args, w):
                     "same_result": bool(torch.equal(out_s, out_ref))}
         ctx_s.close()
 
+    # ---- the step after the round (model update) and the plain-sum rule, timed on their own
+    extras = None
+    if not args.no_extras and rank == 0:
+        extras = {}
+        reps = 3
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def timed(fn):
+            ts = []
+            for _ in range(reps):
+                if flush is not None:
+                    flush.fill_(2)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            return float(np.median(ts))
+
+        weights = torch.zeros((n, w.ld), dtype=torch.float32, device=device)
+        ctx.aggregate(U, out, stream)
+        ctx.apply_update(out, weights, 0.01, stream)
+        ms = timed(lambda: ctx.apply_update(out, weights, 0.01, stream))
+        alg = 8 * n * d + 4 * n * ((d + 31) // 32)
+        extras["model_update"] = {"ms": ms, "algorithmic_gbs": alg / (ms * 1e-3) / 1e9, "elements_per_s": n * d / (ms * 1e-3)}
+        del weights
+        ctx_sum = B.Brace(n, f, d, B.default_params(rule=B.RULE_SUM, agg_mode=B.AGG_FUSED), device=device)
+        out_sum = ctx_sum.new_output(device=device)
+        ctx_sum.aggregate(U, out_sum, stream)
+        ms = timed(lambda: ctx_sum.aggregate(U, out_sum, stream))
+        alg = 8 * n * d + 2 * 4 * d
+        extras["sum_rule_fused"] = {"ms": ms, "algorithmic_gbs": alg / (ms * 1e-3) / 1e9, "elements_per_s": n * d / (ms * 1e-3)}
+        ctx_sum.close()
+        del out_sum
+        torch.cuda.empty_cache()
+
     if rank != 0:
         return
     peaks, peak_kind = measured_peaks()
@@ -370,7 +406,7 @@ def run_cuda(args, w):
         "roofline": roofline, "cpu_baseline": cpu_baseline,
         "phases_ms": {"inject": inj_avg_ms, "aggregate": agg_avg_ms},
         "aggregate_only_elements_per_s": n * d / (agg_avg_ms * 1e-3),
-        "stepwise": stepwise,
+        "stepwise": stepwise, "extras": extras,
     }
     print(json.dumps(line), flush=True)
     ctx.close()
@@ -415,6 +451,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-stepwise", action="store_true")
+    ap.add_argument("--no-extras", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3

@@ -204,6 +204,20 @@ int brace_ring_allgather_step(brace_ctx* ctx, int32_t step, void* d_out, int64_t
 int brace_aggregate(brace_ctx* ctx, const float* d_updates, int64_t ld, void* d_out, int64_t out_ld,
                     brace_stream_t stream);
 
+/* The step after a round: every client applies the aggregate it now holds to
+ * its own parameter vector (row c of d_weights [n][ld_weights] float32,
+ * updated in place; ld_weights >= d).
+ *   sign rules: w_c[k] <- w_c[k] - eta * (+1 or -1 read from row c of d_out)
+ *     (Appendix A, update rule: no 1/n, the aggregate has unit entries);
+ *   SUM: w_c[k] <- w_c[k] - (eta / n) * sum[k]  (Section 2.2, per-client update
+ *     after plain ring-all-reduce); with params.mean the rows already hold the
+ *     mean and the factor is eta.
+ * float32 arithmetic, each operation rounded to nearest.  d_out / out_ld as for
+ * brace_aggregate; it is only read.  Errors: INVALID_ARG (null, short rows,
+ * non-finite eta), WORKSPACE, CUDA. */
+int brace_apply_update(brace_ctx* ctx, const void* d_out, int64_t out_ld, float* d_weights,
+                       int64_t ld_weights, float eta, brace_stream_t stream);
+
 /* Same round with HOST inputs and outputs: copies h_updates [n][ld] to the
  * caller's device staging matrix d_updates_stage [n][ld], applies `attack`
  * there if attack != NULL (attack->noise / uniform are HOST [f][*_ld] matrices,

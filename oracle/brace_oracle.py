@@ -305,6 +305,27 @@ def sum_direct_f64(updates: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
+# The model update that follows a round
+# --------------------------------------------------------------------------
+def apply_update(weights: np.ndarray, outputs: np.ndarray, eta: float, rule: int, mean: bool = False) -> np.ndarray:
+    """Per-client parameter update, in float64.
+
+    Plain RAR (Section 2.2): w_i <- w_i - (eta / n) * sum_j g_j, each client on
+    its own copy; ``outputs`` are the rows the ring left (the sum, or the mean
+    when ``mean``).  Sign rules (Appendix A, update rule): w <- w - eta * (2 I - 1)
+    = w - eta * GAR, no 1/n.  weights, outputs: [n, d].
+    """
+    w = np.asarray(weights, dtype=np.float64)
+    g = np.asarray(outputs, dtype=np.float64)
+    n = w.shape[0]
+    eta64 = np.float64(np.float32(eta))
+    if rule == RULE_SUM:
+        factor = eta64 if mean else eta64 / np.float64(n)
+        return w - factor * g
+    return w - eta64 * g
+
+
+# --------------------------------------------------------------------------
 # Section 2.2 / Section 3 / Table 1: bits each client sends per round
 # --------------------------------------------------------------------------
 def sent_bits(trace: RingTrace, m_bits: int, rule: int) -> np.ndarray:

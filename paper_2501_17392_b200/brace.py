@@ -57,6 +57,7 @@ SIGNATURES = {
     "brace_consensus": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
     "brace_ring_allgather_step": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p]),
     "brace_aggregate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p]),
+    "brace_apply_update": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_float, C.c_void_p]),
     "brace_aggregate_host": (C.c_int, [C.c_void_p, C.POINTER(Attack), C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "brace_debug_mailbox": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_int64),
@@ -241,6 +242,14 @@ class Brace:
 
     def aggregate(self, updates: torch.Tensor, out: torch.Tensor, stream=None):
         _check(self.aggregate_status(updates, out, stream), "brace_aggregate")
+
+    def apply_update_status(self, out: torch.Tensor, weights: torch.Tensor, eta: float, stream=None) -> int:
+        return lib().brace_apply_update(self._ctx, _ptr(out), out.stride(0), _ptr(weights), weights.stride(0),
+                                        float(eta), _stream(stream))
+
+    def apply_update(self, out: torch.Tensor, weights: torch.Tensor, eta: float, stream=None):
+        """Each client's parameter row moves by the aggregate in its output row."""
+        _check(self.apply_update_status(out, weights, eta, stream), "brace_apply_update")
 
     def aggregate_host(self, attack: Attack | None, h_updates: torch.Tensor, h_out: torch.Tensor,
                        d_updates: torch.Tensor, d_out: torch.Tensor, d_noise=None, d_uniform=None, stream=None):

@@ -660,6 +660,38 @@ int brace_quantize(brace_ctx* ctx, const float* d_updates, int64_t ld, int8_t* d
   return check_launch(ctx);
 }
 
+int brace_apply_update(brace_ctx* ctx, const void* d_out, int64_t out_ld, float* d_weights, int64_t ld_weights,
+                       float eta, brace_stream_t stream) {
+  int rc = check_device_ctx(ctx);
+  if (rc != BRACE_OK) return rc;
+  rc = check_out(ctx, d_out, out_ld);
+  if (rc != BRACE_OK) return rc;
+  if (!d_weights || ld_weights < ctx->d || !std::isfinite(eta)) return BRACE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_weights) & 3u) != 0) return BRACE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  dim3 grid(tiles(ctx->d, kThreads * 4), (unsigned)ctx->n);
+  const bool wvec = (ld_weights % 4 == 0) && aligned16(d_weights);
+  if (ctx->p.rule == BRACE_RULE_SUM) {
+    // the rows hold the sum (or already the mean): w <- w - (eta/n) * sum, or w - eta * mean
+    const float scale = ctx->p.mean ? eta : eta / (float)ctx->n;
+    const bool vec = wvec && (out_ld % 4 == 0) && aligned16(d_out);
+    if (vec)
+      apply_update_f32_kernel<true><<<grid, kThreads, 0, st>>>((const float*)d_out, out_ld, d_weights, ld_weights,
+                                                              ctx->d, scale);
+    else
+      apply_update_f32_kernel<false><<<grid, kThreads, 0, st>>>((const float*)d_out, out_ld, d_weights, ld_weights,
+                                                               ctx->d, scale);
+  } else {
+    if (wvec)
+      apply_update_bits_kernel<true><<<grid, kThreads, 0, st>>>((const uint32_t*)d_out, out_ld, d_weights,
+                                                               ld_weights, ctx->d, eta);
+    else
+      apply_update_bits_kernel<false><<<grid, kThreads, 0, st>>>((const uint32_t*)d_out, out_ld, d_weights,
+                                                                ld_weights, ctx->d, eta);
+  }
+  return check_launch(ctx);
+}
+
 int brace_ring_reduce_scatter_step(brace_ctx* ctx, int32_t step, const float* d_updates, int64_t ld,
                                    brace_stream_t stream) {
   int rc = check_device_ctx(ctx);

@@ -543,6 +543,55 @@ fused_sum_kernel(const FusedArgs a) {
 }
 
 // ---------------------------------------------------------------------------
+// Model update that follows a round: each client applies the aggregate it holds
+// to its own parameter row.  Sign rules (Appendix A, update rule): w <- w - eta*(+-1);
+// plain ring-all-reduce (Section 2.2): w <- w - scale*sum with scale = eta/n.
+// grid = (tiles over d, n clients); 4 coordinates per thread.
+// ---------------------------------------------------------------------------
+template <bool VEC>
+__global__ void __launch_bounds__(256)
+apply_update_bits_kernel(const uint32_t* __restrict__ out, int64_t out_ld, float* __restrict__ Wt, int64_t ld_w,
+                         int64_t d, float eta) {
+  const int c = blockIdx.y;
+  const int64_t k = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (k >= d) return;
+  const uint32_t nib = (__ldg(out + (int64_t)c * out_ld + (k >> 5)) >> (int)(k & 31)) & 0xFu;
+  float* w = Wt + (int64_t)c * ld_w + k;
+  if (VEC && k + 4 <= d) {
+    float4 v = *reinterpret_cast<float4*>(w);
+    v.x = __fsub_rn(v.x, (nib & 1u) ? eta : -eta);
+    v.y = __fsub_rn(v.y, (nib & 2u) ? eta : -eta);
+    v.z = __fsub_rn(v.z, (nib & 4u) ? eta : -eta);
+    v.w = __fsub_rn(v.w, (nib & 8u) ? eta : -eta);
+    *reinterpret_cast<float4*>(w) = v;
+  } else {
+    for (int q = 0; q < 4 && k + q < d; ++q) w[q] = __fsub_rn(w[q], ((nib >> q) & 1u) ? eta : -eta);
+  }
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(256)
+apply_update_f32_kernel(const float* __restrict__ out, int64_t out_ld, float* __restrict__ Wt, int64_t ld_w,
+                        int64_t d, float scale) {
+  const int c = blockIdx.y;
+  const int64_t k = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (k >= d) return;
+  const float* g = out + (int64_t)c * out_ld + k;
+  float* w = Wt + (int64_t)c * ld_w + k;
+  if (VEC && k + 4 <= d) {
+    const float4 a = ld_stream(g);
+    float4 v = *reinterpret_cast<float4*>(w);
+    v.x = __fsub_rn(v.x, __fmul_rn(scale, a.x));
+    v.y = __fsub_rn(v.y, __fmul_rn(scale, a.y));
+    v.z = __fsub_rn(v.z, __fmul_rn(scale, a.z));
+    v.w = __fsub_rn(v.w, __fmul_rn(scale, a.w));
+    *reinterpret_cast<float4*>(w) = v;
+  } else {
+    for (int q = 0; q < 4 && k + q < d; ++q) w[q] = __fsub_rn(w[q], __fmul_rn(scale, g[q]));
+  }
+}
+
+// ---------------------------------------------------------------------------
 // Phase I on its own (inspection / tests): int8 sign matrix.
 // ---------------------------------------------------------------------------
 template <bool ZS>

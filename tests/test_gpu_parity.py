@@ -233,6 +233,39 @@ def test_other_sign_rules(rule, n, d, G, ld, lam):
     ctxa.close()
 
 
+@pytest.mark.parametrize("rule,mean", [(B.RULE_SIGN_CONSENSUS, 0), (B.RULE_ABS_CONSENSUS, 0), (B.RULE_SUM, 0),
+                                       (B.RULE_SUM, 1)])
+@pytest.mark.parametrize("n,d,ldw", [(8, 100_001, 100_004), (5, 4_099, 4_101), (20, 33_000, 33_024)])
+def test_model_update_after_round(rule, mean, n, d, ldw):
+    """w <- w - eta * aggregate per client; float64 oracle, 1e-5 relative to the larger operand."""
+    g = torch.Generator().manual_seed(n + d)
+    U = torch.zeros((n, d + 3), dtype=torch.float32)
+    U[:, :d].normal_(generator=g)
+    Wt = torch.zeros((n, ldw), dtype=torch.float32)
+    Wt.normal_(generator=g)
+    eta = 0.03
+    Uh, Wh = U.numpy()[:, :d], Wt.numpy().copy()
+    tr = O.ring_round(Uh, rule=rule, lam=1.0, mean=bool(mean), keep_states=False)
+    exp = O.apply_update(Wh[:, :d], tr.outputs, eta, rule, mean=bool(mean))
+    ctx = B.Brace(n, 0, d, B.default_params(rule=rule, lam=1.0, mean=mean, agg_mode=B.AGG_STEPWISE))
+    out = ctx.new_output()
+    ctx.aggregate(U.cuda(), out)
+    Wd = Wt.cuda()
+    ctx.apply_update(out, Wd, eta)
+    got = Wd.cpu().numpy()
+    scale = np.maximum(np.abs(exp), np.abs(Wh[:, :d].astype(np.float64)))
+    assert (np.abs(got[:, :d] - exp) <= REL_TOL * scale + 1e-30).all()
+    assert np.array_equal(got[:, d:], Wh[:, d:])                       # row padding untouched
+    if rule != B.RULE_SUM:                                             # one exact float32 subtraction of +-eta
+        e32 = np.float32(eta)
+        ref32 = Wh[:, :d] - e32 * tr.outputs.astype(np.float32)
+        assert np.array_equal(got[:, :d].view(np.uint32), ref32.view(np.uint32))
+    assert B.lib().brace_apply_update(ctx._ctx, out.data_ptr(), out.stride(0), Wd.data_ptr(), d - 1, eta,
+                                      None) == B.ERR_INVALID_ARG   # rows shorter than d
+    assert ctx.apply_update_status(out, Wd, float("nan")) == B.ERR_INVALID_ARG
+    ctx.close()
+
+
 def test_unaligned_rows_fall_back_to_scalar_kernels():
     """Row stride not a multiple of 4 and a base pointer off 16 bytes."""
     n, d, ld = 6, 3_001, 3_003

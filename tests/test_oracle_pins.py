@@ -417,3 +417,30 @@ def test_abs_consensus_is_symmetric_and_is_the_union_of_both_directions():
     for rule in (O.RULE_MAJORITY_SIGN, O.RULE_ABS_CONSENSUS):
         tr = O.ring_round(V, rule=rule, lam=1, granule=1, keep_states=False)
         assert O.sent_bits(tr, 8, rule).tolist() == [54] * 4      # Table 1 row n=4, d=8, m=8
+
+
+# ---------------------------------------------------------------- the model update after a round
+def test_apply_update_closed_forms(golden):
+    g = golden("rar_worked_example.txt")
+    U = _mat(g["g1"], g["g2"], g["g3"])
+    tr = O.ring_round(U, rule=O.RULE_SUM, granule=1)
+    w0 = np.zeros((3, 3), dtype=np.float32)
+    # Section 2.2: w - (eta / n) * sum; with eta = n = 3 and w = 0 every client lands on -sum
+    w1 = O.apply_update(w0, tr.outputs, 3.0, O.RULE_SUM)
+    assert w1.tolist() == [[-22, -1, -5]] * 3
+    trm = O.ring_round(U, rule=O.RULE_SUM, granule=1, mean=True)
+    assert np.allclose(O.apply_update(w0, trm.outputs, 3.0, O.RULE_SUM, mean=True), np.array([[-22, -1, -5]] * 3),
+                       rtol=1e-6)
+    # Appendix A: BRACE moves every coordinate by exactly eta, against the aggregate's sign, no 1/n
+    rng = np.random.default_rng(12)
+    n, d, eta = 6, 500, 0.125
+    V = rng.standard_normal((n, d)).astype(np.float32)
+    w = rng.standard_normal((n, d)).astype(np.float32)
+    tb = O.ring_round(V, lam=1, granule=16, keep_states=False)
+    w2 = O.apply_update(w, tb.outputs, eta, O.RULE_SIGN_CONSENSUS)
+    assert np.array_equal(np.abs(w2 - w.astype(np.float64)), np.full((n, d), eta))
+    assert np.array_equal(np.sign(w.astype(np.float64) - w2), tb.outputs.astype(np.float64))
+    # identical starting points stay identical across clients (all clients hold the same aggregate)
+    same = np.tile(w[0], (n, 1))
+    w3 = O.apply_update(same, tb.outputs, eta, O.RULE_SIGN_CONSENSUS)
+    assert (w3 == w3[0]).all()
