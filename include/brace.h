@@ -229,6 +229,28 @@ int brace_aggregate_host(brace_ctx* ctx, const brace_attack* attack, const float
                          void* h_out, int64_t out_ld, float* d_updates_stage, float* d_noise_stage,
                          float* d_uniform_stage, void* d_out_stage, brace_stream_t stream);
 
+/* Bits each client sends in one round, from this context's actual partition
+ * (Section 2.2 and Section 3 cost paragraphs, Table 1).  m_bits = width of one
+ * gradient coordinate on the wire (the paper's m).  Host only.
+ *   sc_bits               m*n*d (server-client)
+ *   rar_bits_min/max      plain ring-all-reduce: client c sends every sub-vector but (c+1) mod n during
+ *                         share-reduce and every one but (c+2) mod n during share-only, m bits per coordinate;
+ *                         closed form 2*m*d*(n-1)/n when n divides d
+ *   brace_bits_min/max    sign rules: the same share-reduce at m bits, share-only at 1 bit per coordinate;
+ *                         closed form d*(n-1)*(m+1)/n
+ *   packed_bits_min/max   as brace_bits with share-reduce at the width the mailboxes really use
+ *   partial_bits_used     8 or 16 (mailbox entry width); partial_bits_min = ceil(log2(2n+1)), the fewest
+ *                         bits that can hold a partial sign-sum in [-n, n]                                 */
+typedef struct brace_cost {
+  int64_t sc_bits;
+  int64_t rar_bits_min, rar_bits_max;
+  int64_t brace_bits_min, brace_bits_max;
+  int64_t packed_bits_min, packed_bits_max;
+  double rar_closed_form, brace_closed_form;
+  int32_t partial_bits_used, partial_bits_min;
+} brace_cost;
+int brace_comm_cost(const brace_ctx* ctx, int32_t m_bits, brace_cost* cost);
+
 /* Test aid: device pointer, length (entries) and sub-vector id of the mailbox
  * that client `client` filled at the most recent share-reduce hop
  * (hops_back = 0) or at the hop before it (hops_back = 1; the other mailbox

@@ -32,6 +32,13 @@ class Attack(C.Structure):
                 ("noise_ld", C.c_int64), ("uniform", C.c_void_p), ("uniform_ld", C.c_int64)]
 
 
+class Cost(C.Structure):
+    _fields_ = [("sc_bits", C.c_int64), ("rar_bits_min", C.c_int64), ("rar_bits_max", C.c_int64),
+                ("brace_bits_min", C.c_int64), ("brace_bits_max", C.c_int64), ("packed_bits_min", C.c_int64),
+                ("packed_bits_max", C.c_int64), ("rar_closed_form", C.c_double), ("brace_closed_form", C.c_double),
+                ("partial_bits_used", C.c_int32), ("partial_bits_min", C.c_int32)]
+
+
 class BraceError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -50,6 +57,7 @@ SIGNATURES = {
     "brace_destroy": (C.c_int, [C.c_void_p]),
     "brace_segment": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "brace_last_cuda_error": (C.c_int, [C.c_void_p]),
+    "brace_comm_cost": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(Cost)]),
     "brace_inject_attack": (C.c_int, [C.c_void_p, C.POINTER(Attack), C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                       C.c_void_p]),
     "brace_quantize": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p]),
@@ -190,6 +198,11 @@ class Brace:
         b, e = C.c_int64(), C.c_int64()
         _check(lib().brace_segment(self._ctx, j, C.byref(b), C.byref(e)), "brace_segment")
         return b.value, e.value
+
+    def comm_cost(self, m_bits: int) -> Cost:
+        cost = Cost()
+        _check(lib().brace_comm_cost(self._ctx, m_bits, C.byref(cost)), "brace_comm_cost")
+        return cost
 
     def last_cuda_error(self) -> int:
         return int(lib().brace_last_cuda_error(self._ctx))

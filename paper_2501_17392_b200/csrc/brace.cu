@@ -620,6 +620,34 @@ int brace_segment(const brace_ctx* ctx, int32_t j, int64_t* begin, int64_t* end)
   return BRACE_OK;
 }
 
+int brace_comm_cost(const brace_ctx* ctx, int32_t m_bits, brace_cost* cost) {
+  if (!ctx || !cost || m_bits < 1) return BRACE_ERR_INVALID_ARG;
+  const int n = ctx->n;
+  const int64_t d = ctx->d, m = m_bits;
+  const int used = ctx->p.rule == BRACE_RULE_SUM ? 32 : 8 * ctx->entry_bytes;
+  int need = 1;
+  while ((1LL << need) < 2LL * n + 1) ++need;
+  std::memset(cost, 0, sizeof(*cost));
+  cost->sc_bits = m * n * d;
+  cost->rar_closed_form = 2.0 * (double)m * (double)d * (double)(n - 1) / (double)n;
+  cost->brace_closed_form = (double)d * (double)(n - 1) * (double)(m + 1) / (double)n;
+  cost->partial_bits_used = used;
+  cost->partial_bits_min = need;
+  for (int c = 0; c < n; ++c) {
+    const int skip_rs = (c + 1) % n, skip_ag = (c + 2) % n;   // the sub-vectors client c never sends
+    const int64_t rs = d - (seg_end(ctx->pt, skip_rs) - ctx->pt.begin(skip_rs));
+    const int64_t ag = d - (seg_end(ctx->pt, skip_ag) - ctx->pt.begin(skip_ag));
+    const int64_t rar = (rs + ag) * m, brace_bits = rs * m + ag, packed = rs * used + ag;
+    if (c == 0 || rar < cost->rar_bits_min) cost->rar_bits_min = rar;
+    if (c == 0 || rar > cost->rar_bits_max) cost->rar_bits_max = rar;
+    if (c == 0 || brace_bits < cost->brace_bits_min) cost->brace_bits_min = brace_bits;
+    if (c == 0 || brace_bits > cost->brace_bits_max) cost->brace_bits_max = brace_bits;
+    if (c == 0 || packed < cost->packed_bits_min) cost->packed_bits_min = packed;
+    if (c == 0 || packed > cost->packed_bits_max) cost->packed_bits_max = packed;
+  }
+  return BRACE_OK;
+}
+
 int brace_last_cuda_error(const brace_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
 
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid) {

@@ -112,3 +112,35 @@ def test_host_only_context_refuses_device_calls():
     assert lib.brace_aggregate(None, 4096, 100, 4096, 4, None) == B.ERR_INVALID_ARG
     assert ctx.last_cuda_error() == 0
     ctx.close()
+
+
+def test_comm_cost_matches_table1_and_the_oracle_schedule(golden):
+    """Table 1 closed forms when n divides d (G = 1); otherwise the per-client
+    counts of the oracle's simulated schedule."""
+    import numpy as np
+    for n, d, m, sc, rar, brace in golden("comm_cost_table1.txt")["rows"]:
+        ctx = B.Brace(n, 0, d, B.default_params(granule=1), host_only=True)
+        c = ctx.comm_cost(m)
+        assert c.sc_bits == sc
+        assert c.rar_bits_min == c.rar_bits_max == rar and c.rar_closed_form == rar
+        assert c.brace_bits_min == c.brace_bits_max == brace and c.brace_closed_form == brace
+        assert c.partial_bits_used == 8
+        assert 2 ** c.partial_bits_min >= 2 * n + 1 > 2 ** (c.partial_bits_min - 1)
+        ctx.close()
+    rng = np.random.default_rng(0)
+    for n, d, G in [(5, 23, 1), (7, 1000, 32), (16, 300, 128), (8, 100_000, 128)]:
+        U = rng.standard_normal((n, d)).astype(np.float32)
+        tr = O.ring_round(U, lam=0, granule=G, keep_states=False)
+        ctx = B.Brace(n, 0, d, B.default_params(granule=G), host_only=True)
+        c = ctx.comm_cost(32)
+        bits = O.sent_bits(tr, 32, O.RULE_SIGN_CONSENSUS)
+        assert (c.brace_bits_min, c.brace_bits_max) == (int(bits.min()), int(bits.max()))
+        bits = O.sent_bits(tr, 32, O.RULE_SUM)
+        assert (c.rar_bits_min, c.rar_bits_max) == (int(bits.min()), int(bits.max()))
+        bits = O.sent_bits(tr, 8, O.RULE_SIGN_CONSENSUS)
+        assert (c.packed_bits_min, c.packed_bits_max) == (int(bits.min()), int(bits.max()))
+        ctx.close()
+    big = B.Brace(200, 0, 1000, B.default_params(), host_only=True)
+    assert big.comm_cost(32).partial_bits_used == 16 and big.comm_cost(32).partial_bits_min == 9
+    assert B.lib().brace_comm_cost(big._ctx, 0, B.Cost()) == B.ERR_INVALID_ARG
+    big.close()
