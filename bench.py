@@ -316,6 +316,34 @@ def run_cuda(args, w):
         stepwise = {"ms_per_round": ms, "launches_per_round": 2 * (n - 1) + 1,
                     "elements_per_s": n * d / (ms * 1e-3), "algorithmic_gbs": b_ring / (ms * 1e-3) / 1e9,
                     "same_result": bool(torch.equal(out_s, out_ref))}
+        # the same launches replayed from a CUDA graph (removes host launch cost; matters for short hops)
+        try:
+            side = torch.cuda.Stream(device=device)
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                ctx_s.aggregate(U, out_s)
+            stream.wait_stream(side)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                ctx_s.aggregate(U, out_s)
+            graph.replay()
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(reps):
+                if flush is not None:
+                    flush.fill_(1)
+                a.record(stream)
+                graph.replay()
+                b.record(stream)
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            gms = float(np.median(ts))
+            stepwise["graph_ms_per_round"] = gms
+            stepwise["graph_algorithmic_gbs"] = b_ring / (gms * 1e-3) / 1e9
+            stepwise["graph_same_result"] = bool(torch.equal(out_s, out_ref))
+            del graph
+        except RuntimeError as exc:                  # capture unsupported: report, do not fail the bench
+            stepwise["graph_error"] = str(exc)[:200]
         ctx_s.close()
 
     # ---- the step after the round (model update) and the plain-sum rule, timed on their own

@@ -349,6 +349,33 @@ def test_rounds_are_memoryless():
     ctx.close()
 
 
+def test_rounds_can_be_captured_in_a_cuda_graph():
+    """Both round modes enqueue only kernels on the caller's stream, so a stream
+    capture records them; replays on fresh inputs give the oracle's bits."""
+    w = W.scaled(W.WORKLOADS["cfg2"], 70_001)
+    U = W.honest_updates(w, 0, device="cuda")
+    for mode in (B.AGG_FUSED, B.AGG_STEPWISE):
+        ctx = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam, agg_mode=mode))
+        out = ctx.new_output()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            ctx.aggregate(U, out)
+        torch.cuda.current_stream().wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            ctx.aggregate(U, out)
+        for rnd in (1, 2):
+            W.honest_updates(w, rnd, device="cuda", out=U)            # new data in the captured buffer
+            out.fill_(-1)
+            graph.replay()
+            torch.cuda.synchronize()
+            tr = O.ring_round(U.cpu().numpy()[:, :w.d], lam=w.lam, keep_states=False)
+            check_final(out, tr, B.RULE_SIGN_CONSENSUS, w.d)
+        del graph
+        ctx.close()
+
+
 def test_guard_bands_stay_untouched():
     """Canaries around the workspace, the output and the mailbox tails."""
     n, d, ld = 7, 9_001, 9_004
