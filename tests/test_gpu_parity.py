@@ -331,6 +331,43 @@ def test_many_clients_partial_width(n):
         ctx.close()
 
 
+def test_largest_client_count():
+    """n = 32767, the most the int16 partial sums hold: far more clients than granules, so
+    most sub-vectors are empty; unanimous columns reach +-n without wrapping."""
+    import ctypes
+    n, d = 32767, 4096
+    g = torch.Generator().manual_seed(7)
+    U = torch.zeros((n, d), dtype=torch.float32)
+    U.normal_(generator=g)
+    U[:, :32] = 2.0
+    U[:, 32:64] = -2.0
+    Uh = U.numpy()
+    S = O.sign_sum_direct(Uh)
+    assert S[0] == n and S[32] == -n
+    Ud = U.cuda()
+    for rule, lam in ((B.RULE_SIGN_CONSENSUS, float(n - 1)), (B.RULE_SIGN_CONSENSUS, 100.0),
+                      (B.RULE_ABS_CONSENSUS, float(n - 1))):
+        exp = expected_words(O.gar_direct(Uh, lam, rule=rule), d)
+        ctx = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, agg_mode=B.AGG_FUSED))
+        out = ctx.new_output()
+        ctx.aggregate(Ud, out)
+        assert (out_words(out, d) == exp[None, :]).all()
+        ctx.close()
+    # hop by hop: 65 533 launches; the owners' partials are the full sign-sums
+    ctx = B.Brace(n, 0, d, B.default_params(lam=100.0, agg_mode=B.AGG_STEPWISE))
+    out = ctx.new_output()
+    ctx.aggregate(Ud, out)
+    assert (out_words(out, d) == expected_words(O.gar_direct(Uh, 100.0), d)[None, :]).all()
+    for j in (0, 1, 31):
+        b, e = ctx.segment(j)
+        if e > b:
+            seg, box = ctx.mailbox_tensor((j - 1) % n)
+            assert seg == j and np.array_equal(box.numpy().astype(np.int32), S[b:e])
+    ctx.close()
+    handle = ctypes.c_void_p()
+    assert B.lib().brace_init(ctypes.byref(handle), n + 1, 0, d, B.default_params(), None, 0, None) == B.ERR_UNSUPPORTED
+
+
 def test_rounds_are_memoryless():
     """Five consecutive rounds on one context equal five rounds on fresh contexts."""
     w = W.scaled(W.WORKLOADS["cfg5"], 40_000)
