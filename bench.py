@@ -381,6 +381,26 @@ def run_cuda(args, w):
         ctx_sum.close()
         del out_sum
         torch.cuda.empty_cache()
+        if n <= 128:
+            # coordinate-wise median / trimmed mean: arithmetic-bound (bitonic network of min/max pairs on the
+            # ALU pipe: 64 lanes per clock per SM, 148 SMs, at the maximum SM clock of the peaks file)
+            res = torch.empty(d, dtype=torch.float32, device=device)
+            npad = 4
+            while npad < n:
+                npad *= 2
+            lg = npad.bit_length() - 1
+            alu_ops = 2 * (npad * lg * (lg + 1) // 4)                    # min + max per compare-exchange
+            peaks_now, _ = measured_peaks()
+            alu_peak = 148 * 64 * peaks_now.get("sm_max_mhz", 1965.0) * 1e6
+            for label, kind, trim in (("median", B.STAT_MEDIAN, 0), ("trimmed_mean", B.STAT_TRIMMED_MEAN, f)):
+                ctx.coordinate_stat(kind, trim, U, res, stream)
+                ms = timed(lambda: ctx.coordinate_stat(kind, trim, U, res, stream))
+                extras["coordinate_" + label] = {
+                    "ms": ms, "elements_per_s": n * d / (ms * 1e-3), "bound": "alu",
+                    "alu_ops_per_coordinate": alu_ops, "achieved_ops_per_s": alu_ops * d / (ms * 1e-3),
+                    "peak_ops_per_s": alu_peak, "frac": alu_ops * d / (ms * 1e-3) / alu_peak,
+                    "hbm_gbs": (4 * n * d + 4 * d) / (ms * 1e-3) / 1e9}
+            del res
 
     if rank != 0:
         return

@@ -218,6 +218,24 @@ int brace_aggregate(brace_ctx* ctx, const float* d_updates, int64_t ld, void* d_
 int brace_apply_update(brace_ctx* ctx, const void* d_out, int64_t out_ld, float* d_weights,
                        int64_t ld_weights, float eta, brace_stream_t stream);
 
+/* Coordinate-wise statistics over the n client values of every coordinate: the
+ * server-side aggregation rules the paper compares against (Section 5.1: Median,
+ * Trimmed-mean).  They need all n slices of a coordinate at once, so they are
+ * not ring rules (Section 3); this call reads d_updates [n][ld] directly and
+ * writes ONE vector d_result [d] float32.  It uses no workspace (a host-only
+ * context is accepted).
+ *   BRACE_STAT_MEDIAN        the middle value of the n sorted values; for even n
+ *                            the mean of the two middle values (float64 add and
+ *                            halve, rounded once to float32); `trim` is ignored
+ *   BRACE_STAT_TRIMMED_MEAN  drop the `trim` smallest and the `trim` largest
+ *                            values (0 <= 2*trim < n), then the mean of the rest,
+ *                            summed in float64 in ascending order and rounded once
+ * +-Inf take part in the ordering; a NaN input makes that coordinate's result
+ * unspecified.  n <= 128 (else BRACE_ERR_UNSUPPORTED). */
+enum { BRACE_STAT_MEDIAN = 0, BRACE_STAT_TRIMMED_MEAN = 1 };
+int brace_coordinate_stat(brace_ctx* ctx, int32_t kind, int32_t trim, const float* d_updates, int64_t ld,
+                          float* d_result, brace_stream_t stream);
+
 /* Same round with HOST inputs and outputs: copies h_updates [n][ld] to the
  * caller's device staging matrix d_updates_stage [n][ld], applies `attack`
  * there if attack != NULL (attack->noise / uniform are HOST [f][*_ld] matrices,

@@ -305,6 +305,37 @@ def sum_direct_f64(updates: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
+# Section 5.1: the server-side coordinate-wise rules BRACE is compared with
+# --------------------------------------------------------------------------
+def coordinate_median(updates: np.ndarray) -> np.ndarray:
+    """Coordinate-wise median of the n client values: the middle one of the n
+    sorted values, for even n the mean of the two middle ones (float64), rounded
+    to float32."""
+    srt = np.sort(np.asarray(updates, dtype=np.float32), axis=0)
+    n = srt.shape[0]
+    if n % 2 == 1:
+        return srt[n // 2]
+    lo, hi = srt[n // 2 - 1].astype(np.float64), srt[n // 2].astype(np.float64)
+    with np.errstate(invalid="ignore"):
+        return (0.5 * (lo + hi)).astype(np.float32)
+
+
+def coordinate_trimmed_mean(updates: np.ndarray, trim: int) -> np.ndarray:
+    """Coordinate-wise trimmed mean: per coordinate drop the ``trim`` smallest and
+    the ``trim`` largest of the n values and average the rest (summed in float64
+    in ascending order, one rounding to float32)."""
+    srt = np.sort(np.asarray(updates, dtype=np.float32), axis=0)
+    n = srt.shape[0]
+    if trim < 0 or 2 * trim >= n:
+        raise ValueError("need 0 <= 2*trim < n")
+    acc = np.zeros(srt.shape[1], dtype=np.float64)
+    with np.errstate(invalid="ignore"):                 # +Inf and -Inf in one column give NaN, as they should
+        for i in range(trim, n - trim):
+            acc = acc + srt[i].astype(np.float64)
+    return (acc / np.float64(n - 2 * trim)).astype(np.float32)
+
+
+# --------------------------------------------------------------------------
 # The model update that follows a round
 # --------------------------------------------------------------------------
 def apply_update(weights: np.ndarray, outputs: np.ndarray, eta: float, rule: int, mean: bool = False) -> np.ndarray:

@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libbrace.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BAD_STEP, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
 RULE_SIGN_CONSENSUS, RULE_SUM, RULE_MAJORITY_SIGN, RULE_ABS_CONSENSUS = 0, 1, 2, 3
 AGG_AUTO, AGG_STEPWISE, AGG_FUSED = 0, 1, 2
+STAT_MEDIAN, STAT_TRIMMED_MEAN = 0, 1
 ATTACK_NONE, ATTACK_SCALE_OWN, ATTACK_GAUSSIAN, ATTACK_SCALED_MEAN, ATTACK_MEAN_SHIFT, ATTACK_SPARSE_NOISE = range(6)
 
 
@@ -66,6 +67,8 @@ SIGNATURES = {
     "brace_ring_allgather_step": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p]),
     "brace_aggregate": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p]),
     "brace_apply_update": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_float, C.c_void_p]),
+    "brace_coordinate_stat": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p,
+                                        C.c_void_p]),
     "brace_aggregate_host": (C.c_int, [C.c_void_p, C.POINTER(Attack), C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "brace_debug_mailbox": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_int64),
@@ -263,6 +266,15 @@ class Brace:
     def apply_update(self, out: torch.Tensor, weights: torch.Tensor, eta: float, stream=None):
         """Each client's parameter row moves by the aggregate in its output row."""
         _check(self.apply_update_status(out, weights, eta, stream), "brace_apply_update")
+
+    def coordinate_stat_status(self, kind: int, trim: int, updates: torch.Tensor, result: torch.Tensor,
+                               stream=None) -> int:
+        return lib().brace_coordinate_stat(self._ctx, kind, trim, _ptr(updates), updates.stride(0), _ptr(result),
+                                           _stream(stream))
+
+    def coordinate_stat(self, kind: int, trim: int, updates: torch.Tensor, result: torch.Tensor, stream=None):
+        """Coordinate-wise median / trimmed mean of the n rows into one float32 vector."""
+        _check(self.coordinate_stat_status(kind, trim, updates, result, stream), "brace_coordinate_stat")
 
     def aggregate_host(self, attack: Attack | None, h_updates: torch.Tensor, h_out: torch.Tensor,
                        d_updates: torch.Tensor, d_out: torch.Tensor, d_noise=None, d_uniform=None, stream=None):

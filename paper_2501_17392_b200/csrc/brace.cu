@@ -720,6 +720,29 @@ int brace_apply_update(brace_ctx* ctx, const void* d_out, int64_t out_ld, float*
   return check_launch(ctx);
 }
 
+int brace_coordinate_stat(brace_ctx* ctx, int32_t kind, int32_t trim, const float* d_updates, int64_t ld,
+                          float* d_result, brace_stream_t stream) {
+  if (!ctx) return BRACE_ERR_INVALID_ARG;
+  int rc = check_updates(ctx, d_updates, ld);
+  if (rc != BRACE_OK) return rc;
+  if (!d_result || (kind != BRACE_STAT_MEDIAN && kind != BRACE_STAT_TRIMMED_MEAN)) return BRACE_ERR_INVALID_ARG;
+  if (kind == BRACE_STAT_TRIMMED_MEAN && (trim < 0 || 2 * (int64_t)trim >= ctx->n)) return BRACE_ERR_INVALID_ARG;
+  if (ctx->n > 128) return BRACE_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const unsigned blocks = tiles(ctx->d, 128);
+  const int n = ctx->n;
+#define BRACE_STAT(NP) \
+  coordinate_stat_kernel<NP><<<blocks, 128, 0, st>>>(kind, trim, n, d_updates, ld, d_result, ctx->d)
+  if (n <= 4) BRACE_STAT(4);
+  else if (n <= 8) BRACE_STAT(8);
+  else if (n <= 16) BRACE_STAT(16);
+  else if (n <= 32) BRACE_STAT(32);
+  else if (n <= 64) BRACE_STAT(64);
+  else BRACE_STAT(128);
+#undef BRACE_STAT
+  return check_launch(ctx);
+}
+
 int brace_ring_reduce_scatter_step(brace_ctx* ctx, int32_t step, const float* d_updates, int64_t ld,
                                    brace_stream_t stream) {
   int rc = check_device_ctx(ctx);

@@ -890,4 +890,60 @@ inject_stats_reg_kernel(int kind, const __grid_constant__ HonestRows rows, const
   for (int bq = 0; bq < f; ++bq) Uo[(int64_t)ids[bq] * ld_u + k] = v;
 }
 
+// ---------------------------------------------------------------------------
+// Coordinate-wise median / trimmed mean over the n client values of each
+// coordinate (the server-side rules Section 5.1 compares against; they need all
+// n slices at once, which is why they cannot run inside the ring, Section 3).
+// A thread owns one coordinate: its n values are loaded into registers, padded
+// with +Inf to NP (a power of two) and sorted by a fully unrolled bitonic
+// network of min/max pairs; the statistic is then read off the sorted registers.
+// Arithmetic-bound: NP*log2(NP)*(log2(NP)+1)/4 compare-exchanges per coordinate.
+// ---------------------------------------------------------------------------
+template <int NP>
+__global__ void __launch_bounds__(128)
+coordinate_stat_kernel(int kind, int trim, int n, const float* __restrict__ U, int64_t ld, float* __restrict__ res,
+                       int64_t d) {
+  const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= d) return;
+  const float* src = U + k;
+  float x[NP];
+#pragma unroll
+  for (int i = 0; i < NP; ++i) x[i] = (i < n) ? __ldcs(src + (int64_t)i * ld) : __int_as_float(0x7f800000);
+  // bitonic sort, ascending
+#pragma unroll
+  for (int size = 2; size <= NP; size <<= 1) {
+#pragma unroll
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+#pragma unroll
+      for (int i = 0; i < NP; ++i) {
+        const int l = i ^ stride;
+        if (l > i) {
+          const float a = x[i], b = x[l];
+          const float lo = fminf(a, b), hi = fmaxf(a, b);
+          if ((i & size) == 0) { x[i] = lo; x[l] = hi; }
+          else                 { x[i] = hi; x[l] = lo; }
+        }
+      }
+    }
+  }
+  float out;
+  if (kind == 0) {                                   // median: middle value, or the mean of the two middle ones
+    const int hi_idx = n >> 1, lo_idx = (n - 1) >> 1;
+    float vlo = 0.f, vhi = 0.f;
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+      if (i == lo_idx) vlo = x[i];
+      if (i == hi_idx) vhi = x[i];
+    }
+    out = (lo_idx == hi_idx) ? vlo : __double2float_rn(__dmul_rn(0.5, __dadd_rn((double)vlo, (double)vhi)));
+  } else {                                           // trimmed mean: drop `trim` smallest and largest, float64 mean
+    double acc = 0.0;
+#pragma unroll
+    for (int i = 0; i < NP; ++i)
+      if (i >= trim && i < n - trim) acc = __dadd_rn(acc, (double)x[i]);
+    out = __double2float_rn(__ddiv_rn(acc, (double)(n - 2 * trim)));
+  }
+  res[k] = out;
+}
+
 }  // namespace brace

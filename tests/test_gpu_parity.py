@@ -266,6 +266,45 @@ def test_model_update_after_round(rule, mean, n, d, ldw):
     ctx.close()
 
 
+@pytest.mark.parametrize("n", [2, 3, 4, 5, 8, 9, 16, 20, 33, 64, 65, 100, 128])
+def test_coordinate_median_and_trimmed_mean(n):
+    """The server-side coordinate-wise rules: sorted in registers, same bits as the oracle's
+    sort + ascending float64 sum."""
+    d, ld = 6_001, 6_003
+    g = torch.Generator().manual_seed(n)
+    U = torch.zeros((n, ld), dtype=torch.float32)
+    U[:, :d].normal_(generator=g)
+    U[:, :d][torch.rand((n, d), generator=g) < 0.1] = 0.0
+    U[0, :50] = float("inf")
+    U[n - 1, 25:75] = float("-inf")
+    U[:, 100:110] = 3.25                                              # all clients equal
+    U[:, d:] = float("nan")                                           # padding is never read
+    Uh = U.numpy()[:, :d]
+    ctx = B.Brace(n, 0, d, B.default_params(), host_only=True)        # needs no workspace
+    Ud = U.cuda()
+    res = torch.full((d + 8,), -7.0, dtype=torch.float32, device="cuda")
+    ctx.coordinate_stat(B.STAT_MEDIAN, 0, Ud, res)
+    got = res.cpu().numpy()
+    exp = O.coordinate_median(Uh)
+    assert np.array_equal(got[:d], exp, equal_nan=True)
+    assert (got[d:] == -7.0).all()
+    for trim in sorted({0, 1, n // 5, (n - 1) // 2}):
+        if 2 * trim >= n:
+            continue
+        ctx.coordinate_stat(B.STAT_TRIMMED_MEAN, trim, Ud, res)
+        got = res.cpu().numpy()[:d]
+        exp = O.coordinate_trimmed_mean(Uh, trim)
+        assert np.array_equal(got, exp, equal_nan=True), trim
+    assert ctx.coordinate_stat_status(B.STAT_TRIMMED_MEAN, (n + 1) // 2, Ud, res) == B.ERR_INVALID_ARG
+    assert ctx.coordinate_stat_status(B.STAT_TRIMMED_MEAN, -1, Ud, res) == B.ERR_INVALID_ARG
+    assert ctx.coordinate_stat_status(7, 0, Ud, res) == B.ERR_INVALID_ARG
+    ctx.close()
+    if n == 128:
+        big = B.Brace(129, 0, d, B.default_params(), host_only=True)
+        assert big.coordinate_stat_status(B.STAT_MEDIAN, 0, Ud, res) == B.ERR_UNSUPPORTED
+        big.close()
+
+
 def test_unaligned_rows_fall_back_to_scalar_kernels():
     """Row stride not a multiple of 4 and a base pointer off 16 bytes."""
     n, d, ld = 6, 3_001, 3_003

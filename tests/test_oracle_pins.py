@@ -444,3 +444,37 @@ def test_apply_update_closed_forms(golden):
     same = np.tile(w[0], (n, 1))
     w3 = O.apply_update(same, tb.outputs, eta, O.RULE_SIGN_CONSENSUS)
     assert (w3 == w3[0]).all()
+
+
+# ---------------------------------------------------------------- coordinate-wise median / trimmed mean (Section 5.1)
+def test_coordinate_median_and_trimmed_mean_against_library_routines():
+    from scipy import stats
+    rng = np.random.default_rng(33)
+    for n in (3, 4, 8, 9, 20, 100):
+        U = rng.standard_normal((n, 300)).astype(np.float32)
+        U[rng.random((n, 300)) < 0.1] = 0.0
+        med = O.coordinate_median(U)
+        assert np.allclose(med, np.median(U.astype(np.float64), axis=0), rtol=1e-7, atol=0)
+        for trim in sorted({0, 1, n // 5, (n - 1) // 2}):
+            if 2 * trim >= n:
+                continue
+            tm = O.coordinate_trimmed_mean(U, trim)
+            # scipy cuts int(proportion * n) values from each end of the sorted column
+            ref = stats.trim_mean(U.astype(np.float64), (trim + 0.5) / n, axis=0) if trim else U.astype(np.float64).mean(0)
+            assert np.allclose(tm, ref, rtol=1e-6, atol=1e-9), (n, trim)
+        if n % 2:
+            assert np.array_equal(O.coordinate_trimmed_mean(U, (n - 1) // 2), med)   # all but the middle trimmed
+    # hand-checked columns
+    U = _mat([5, 1, 9, -2], [3, 7, 9, 4], [4, 100, 9, 0], [-6, 2, 9, 8])
+    assert O.coordinate_median(U).tolist() == [3.5, 4.5, 9.0, 2.0]
+    assert O.coordinate_trimmed_mean(U, 1).tolist() == [3.5, 4.5, 9.0, 2.0]
+    assert O.coordinate_trimmed_mean(U, 0).tolist() == [1.5, 27.5, 9.0, 2.5]
+    assert O.coordinate_median(U[:3]).tolist() == [4.0, 7.0, 9.0, 0.0]
+    # order of the clients does not matter; one outlier cannot move the median past its neighbours
+    perm = rng.permutation(4)
+    assert np.array_equal(O.coordinate_median(U[perm]), O.coordinate_median(U))
+    V = U.copy()
+    V[2, 1] = 1e30
+    assert O.coordinate_median(V).tolist() == O.coordinate_median(U).tolist()
+    with pytest.raises(ValueError):
+        O.coordinate_trimmed_mean(U, 2)
