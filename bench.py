@@ -403,6 +403,11 @@ def run_cuda(args, w):
             del res
 
     if rank != 0:
+        # replicas have nothing to report; leave together with rank 0 so that no rank tears the
+        # process group down while another still holds it
+        ctx.close()
+        dist.barrier()
+        dist.destroy_process_group()
         return
     peaks, peak_kind = measured_peaks()
     entry_bytes = 1 if n <= 127 else 2
@@ -463,6 +468,7 @@ def run_cuda(args, w):
     print(json.dumps(line), flush=True)
     ctx.close()
     if world > 1:
+        dist.barrier()
         dist.destroy_process_group()
 
 

@@ -112,6 +112,58 @@ def test_full_size_workload(name):
     torch.cuda.empty_cache()
 
 
+def test_vector_longer_than_2_to_31():
+    """Two clients, d just above 2^31: every in-row offset needs 64-bit arithmetic.
+    Sampled coordinates (head, the 2^31 crossing, sub-vector boundary, tail, random) against Eq. (1),
+    both round modes, plus the attack and model-update kernels at the far end of the rows."""
+    n, d = 2, (1 << 31) + 4_099
+    ld = W.round_up(d, 128)
+    free, _ = torch.cuda.mem_get_info()
+    if free < 3 * n * ld * 4:
+        pytest.skip("not enough free device memory for a 2 x 2^31 float32 matrix")
+    U = torch.empty((n, ld), dtype=torch.float32, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(99)
+    for i in range(n):
+        U[i].normal_(generator=g)
+    ctx = B.Brace(n, 1, d, B.default_params(lam=0.0, agg_mode=B.AGG_FUSED))
+    rng = np.random.default_rng(5)
+    b1, e1 = ctx.segment(1)
+    picks = [np.arange(0, 1024), np.arange((1 << 31) - 600, (1 << 31) + 600), np.arange(b1 - 300, b1 + 300),
+             np.arange(d - 1500, d), rng.integers(0, d, 4096)]
+    idx_np = np.unique(np.concatenate(picks)).astype(np.int64)
+    idx = torch.as_tensor(idx_np, device="cuda")
+    # attack 1 on client 0 (own update scaled), then the round
+    atk = B.make_attack(B.ATTACK_SCALE_OWN, scale=-10.0)
+    Hs = U[:, idx].cpu().numpy()
+    ctx.inject_attack(atk, U, U)
+    Us = U[:, idx].cpu().numpy()
+    exp_u = O.inject_attack(O.ATTACK_SCALE_OWN, Hs, [0], scale=-10.0)
+    assert np.array_equal(Us.view(np.uint32), exp_u.view(np.uint32))
+    out = ctx.new_output()
+    ctx.aggregate(U, out)
+    torch.cuda.synchronize()
+    words = (d + 31) // 32
+    assert torch.equal(out[1, :words], out[0, :words])
+    exp_bits = (O.gar_direct(exp_u, 0.0) > 0).astype(np.int8)
+    assert np.array_equal(bits_at(out[0], idx), exp_bits)
+    assert (int(out[0, words - 1].item()) & 0xFFFFFFFF) >> (d % 32) == 0
+    ctx_s = B.Brace(n, 1, d, B.default_params(lam=0.0, agg_mode=B.AGG_STEPWISE))
+    out_s = ctx_s.new_output()
+    ctx_s.aggregate(U, out_s)
+    torch.cuda.synchronize()
+    assert torch.equal(out_s[:, :words], out[:, :words])
+    # model update in place on the update matrix itself (used here as the parameter rows)
+    before = U[:, idx].cpu().numpy()
+    ctx.apply_update(out, U, 0.5)
+    after = U[:, idx].cpu().numpy()
+    sign = np.where(exp_bits > 0, 1.0, -1.0).astype(np.float32)
+    assert np.array_equal(after, before - np.float32(0.5) * sign[None, :])
+    ctx.close()
+    ctx_s.close()
+    del U, out, out_s
+    torch.cuda.empty_cache()
+
+
 def test_full_size_sum_rule_cfg2():
     """Plain ring-all-reduce at cfg2's size: fused and hop-by-hop give the same
     float32 bits, sampled coordinates match the oracle's ring-order float32 sum."""
