@@ -417,8 +417,10 @@ def run_cuda(args, w):
     words = (d + 31) // 32
     if fused_used:
         agg_alg = algorithmic_bytes_fused(n, d, entry_bytes)
-        agg_kernel = "fused_sign_kernel"
-        launches_per_step = 2
+        spread = n * d >= (1 << 27)                 # the library adds one share-only launch on large problems
+        agg_kernel = "fused_sign_kernel + ag_all_bits_kernel" if spread else "fused_sign_kernel"
+        agg_alg += 4 * words if spread else 0       # the owners' rows are read back once
+        launches_per_step = 3 if spread else 2
     else:
         agg_alg = 4 * n * d + (n - 2) * d + (n - 1) * d + d + 4 * words + (n - 1) * 2 * 4 * words
         agg_kernel = "rs_step_sign_kernel x(n-1) + consensus_sign_kernel + ag_step_bits_kernel x(n-1)"

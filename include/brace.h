@@ -282,8 +282,11 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
  * prefetched) in {(1,8),(2,4),(1,4),(2,8),(1,16)}; fused_grid = 0 launches one
  * CTA per tile, > 0 caps the grid (CTAs then loop over tiles).  Adding 10, 20
  * or 40 to fused_variant makes the share-reduce hop kernel process 1, 2 or 4
- * float4 per thread (default: 4, fewer for short sub-vectors).  Results do not
- * depend on any of these. */
+ * float4 per thread (default: 4, fewer for short sub-vectors).  On large
+ * problems (n*d >= 2^27) the fused kernel writes each sub-vector's bits to its
+ * owner's row and one share-only launch spreads them to the other rows; adding
+ * 1000 forces that at any size, adding 2000 makes the fused kernel write all n
+ * rows itself.  Results do not depend on any of these. */
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid);
 
 /* Bytes of mailbox scratch built into the library for brace_aggregate_static. */

@@ -53,6 +53,7 @@ struct brace_ctx {
   int fused_variant = 0;
   int fused_grid = 0;
   int step_vpt = 0;
+  int spread_mode = 0;   // 0/1 = owner row + share-only launch when the layout allows, 2 = fused kernel writes all rows
   int stats_vw = 0;
 };
 
@@ -285,6 +286,12 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
   a.lam_lo = ctx->lam_lo;
   a.zs = ctx->p.zero_sign;
   a.mean = ctx->p.mean;
+  // sign rules with 16-byte aligned output rows: the kernel writes each sub-vector's bits to its owner's
+  // row and one share-only launch spreads them (long bursts per row instead of 128-byte pieces)
+  // (worth a second launch only on large problems)
+  const bool spread = ctx->p.rule != BRACE_RULE_SUM && (out_ld % 4 == 0) && aligned16(out) && ctx->spread_mode != 2 &&
+                      (ctx->spread_mode == 1 || (int64_t)ctx->n * ctx->d >= (int64_t)1 << 27);
+  a.owner_only = spread ? 1 : 0;
   const bool zs = ctx->p.zero_sign != 0;
   // variant: tile width (float4 per thread per client) x clients prefetched
   int variant = ctx->fused_variant;
@@ -331,6 +338,12 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
   }
 #undef BRACE_FUSED_SIGN
 #undef BRACE_FUSED_SUM
+  int rc = check_launch(ctx);
+  if (rc != BRACE_OK || !spread) return rc;
+  const int rows_per_group = 8;
+  dim3 grid(tiles(ctx->seg_max / 128 + 2, kThreads), (unsigned)ctx->n,
+            (unsigned)((ctx->n + rows_per_group - 1) / rows_per_group));
+  launch_pdl(ag_all_bits_kernel, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, rows_per_group);
   return check_launch(ctx);
 }
 
@@ -652,12 +665,16 @@ int brace_last_cuda_error(const brace_ctx* ctx) { return ctx ? ctx->last_cuda : 
 
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid) {
   if (!ctx || fused_variant < 0 || fused_grid < 0) return BRACE_ERR_INVALID_ARG;
+  const int spread_code = fused_variant / 1000;  // thousands digit: 1 = always spread with a share-only launch, 2 = never
+  fused_variant %= 1000;
   const int stats_code = fused_variant / 100;    // hundreds digit: floats per thread of the statistics kernel
   const int step_code = (fused_variant / 10) % 10;   // tens digit: float4 per thread of the hop kernel
   fused_variant %= 10;
   if (fused_variant > 5 || (step_code != 0 && step_code != 1 && step_code != 2 && step_code != 4) ||
       (stats_code != 0 && stats_code != 1 && stats_code != 2 && stats_code != 4))
     return BRACE_ERR_INVALID_ARG;
+  if (spread_code < 0 || spread_code > 2) return BRACE_ERR_INVALID_ARG;
+  ctx->spread_mode = spread_code;
   ctx->step_vpt = step_code;
   ctx->stats_vw = stats_code;
   ctx->fused_variant = fused_variant;

@@ -52,6 +52,13 @@ __device__ __forceinline__ void store4(int8_t* p, int a, int b, int c, int d) {
 __device__ __forceinline__ void store4(int16_t* p, int a, int b, int c, int d) {
   *reinterpret_cast<short4*>(p) = make_short4((short)a, (short)b, (short)c, (short)d);
 }
+// same, with the streaming hint (written once, not read again by this kernel)
+__device__ __forceinline__ void store4_stream(int8_t* p, int a, int b, int c, int d) {
+  __stcs(reinterpret_cast<char4*>(p), make_char4((signed char)a, (signed char)b, (signed char)c, (signed char)d));
+}
+__device__ __forceinline__ void store4_stream(int16_t* p, int a, int b, int c, int d) {
+  __stcs(reinterpret_cast<short4*>(p), make_short4((short)a, (short)b, (short)c, (short)d));
+}
 __device__ __forceinline__ void load4(const int8_t* p, int& a, int& b, int& c, int& d) {
   char4 v = *reinterpret_cast<const char4*>(p);
   a = v.x; b = v.y; c = v.z; d = v.w;
@@ -289,6 +296,40 @@ ag_step_bits_kernel(Part pt, uint32_t* out, int64_t out_ld, int step) {
   }
 }
 
+// All of Share-Only at once, for the fused round: every sub-vector is copied from
+// its owner's row to the n-1 other rows.  One CTA moves 4 KB of a sub-vector's
+// words (256 threads x 128 bits) to each row in turn, so every row receives long
+// contiguous bursts instead of the 128-byte pieces a tile of the fused kernel
+// could offer.  grid = (chunks over the longest sub-vector, n sub-vectors, groups of rows);
+// needs granule % 128 == 0 and 16-byte aligned rows.
+__global__ void __launch_bounds__(256)
+ag_all_bits_kernel(Part pt, uint32_t* out, int64_t out_ld, int rows_per_group) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int n = pt.n;
+  const int j = blockIdx.y;
+  const int owner = j == 0 ? n - 1 : j - 1;
+  const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+  if (b >= e) return;
+  const int64_t w0 = b >> 5, w1 = (e + 31) >> 5;
+  const int64_t wt = w0 + ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (wt >= w1) return;
+  const int r0 = blockIdx.z * rows_per_group;
+  const int r1 = r0 + rows_per_group < n ? r0 + rows_per_group : n;
+  const uint32_t* src = out + (int64_t)owner * out_ld + wt;
+  if (wt + 4 <= w1) {
+    const uint4 v = *reinterpret_cast<const uint4*>(src);
+    for (int row = r0; row < r1; ++row)
+      if (row != owner) __stcs(reinterpret_cast<uint4*>(out + (int64_t)row * out_ld + wt), v);
+  } else {
+    for (int64_t w = wt; w < w1; ++w) {
+      const uint32_t v = out[(int64_t)owner * out_ld + w];
+      for (int row = r0; row < r1; ++row)
+        if (row != owner) out[(int64_t)row * out_ld + w] = v;
+    }
+  }
+}
+
 template <bool VEC>
 __global__ void __launch_bounds__(256)
 ag_step_f32_kernel(Part pt, float* out, int64_t out_ld, int step) {
@@ -343,6 +384,7 @@ struct FusedArgs {
   int mean;
   int tiles_per_seg;
   int64_t units;
+  int owner_only;   // sign rules: write the consensus bits to the owner's row only (a share-only kernel follows)
 };
 
 template <typename P, int VPT, int UNR, bool ZS>
@@ -407,7 +449,7 @@ fused_sign_kernel(const FusedArgs a) {
 #pragma unroll
             for (int v = 0; v < VPT; ++v) {
               if (nv[v] == 4) {
-                store4(m + off[v], acc[v][0], acc[v][1], acc[v][2], acc[v][3]);
+                store4_stream(m + off[v], acc[v][0], acc[v][1], acc[v][2], acc[v][3]);
               } else {
 #pragma unroll
                 for (int q2 = 0; q2 < 3; ++q2)
@@ -439,7 +481,11 @@ fused_sign_kernel(const FusedArgs a) {
     const int w = tid % WPT;
     if (w < nw) {
       const uint32_t val = sm_words[w];
-      for (int row = tid / WPT; row < n; row += 256 / WPT) out[(int64_t)row * a.out_ld + wb + w] = val;
+      if (a.owner_only) {                            // client j-1 owns sub-vector j (Phase III is local to the owner)
+        if (tid < WPT) out[(int64_t)(j == 0 ? n - 1 : j - 1) * a.out_ld + wb + w] = val;
+      } else {
+        for (int row = tid / WPT; row < n; row += 256 / WPT) out[(int64_t)row * a.out_ld + wb + w] = val;
+      }
     }
     __syncthreads();
   }

@@ -175,7 +175,7 @@ def test_hop_by_hop_and_whole_round(n, d, G, ld, lam, zs, rule):
 
     # (3) whole round, fused kernel, every shape; mailboxes end as the step calls left them
     if fusable:
-        for variant in range(0, 6):
+        for variant in list(range(0, 6)) + [1001, 2001]:  # +1000 / +2000: share-only launch forced / never
             ctxf = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, zero_sign=zs, granule=G, mean=mean,
                                                      agg_mode=B.AGG_FUSED))
             ctxf.workspace.fill_(0x5A)
