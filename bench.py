@@ -491,8 +491,8 @@ def injection_bytes(w):
 # DRAM bytes (read + write) per launch from ncu captures of the full-size workload
 # (profiles/), keyed by (workload, phase); absent where no capture of the current kernel exists.
 TRAFFIC_BYTES: dict = {
-    ("cfg4", "aggregate"): 10_223_567_000 + 328_103_000,   # fused_sign_kernel<int8,1,8>, profiles/fused_sign_kernel_cfg4.md
-    ("cfg4", "inject"): 8_178_284_000 + 1_985_047_000,     # inject_stats_reg_kernel<80>, profiles/inject_stats_reg_kernel_cfg4.md
+    ("cfg4", "aggregate"): 10_222_916_000 + 45_473_000 + 3_302_000 + 254_037_000,   # fused_sign_kernel<int8,1,8> + ag_all_bits_kernel, profiles/fused_sign_kernel_cfg4.md
+    ("cfg4", "inject"): 8_178_365_000 + 1_988_146_000,     # inject_stats_reg_kernel<80>, profiles/inject_stats_reg_kernel_cfg4.md
 }
 
 
