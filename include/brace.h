@@ -98,9 +98,25 @@ typedef struct brace_params {
   int32_t agg_mode;  /* BRACE_AGG_*                                                               */
 } brace_params;
 
-/* Description of one attack.  noise / uniform are [f][*_ld] float32 matrices of
- * standard-normal / uniform[0,1) draws supplied by the caller (row b belongs to
- * the b-th Byzantine id); only the kinds that consume them read them. */
+/* Where the random draws of kinds 2 and 5 come from. */
+enum {
+  BRACE_DRAWS_SUPPLIED = 0, /* the caller passes noise / uniform matrices                          */
+  BRACE_DRAWS_GENERATED = 1 /* the library draws them itself from (seed, round); see below         */
+};
+
+/* Description of one attack.
+ * draws = SUPPLIED: noise / uniform are [f][*_ld] float32 matrices of standard-normal /
+ * uniform[0,1) draws supplied by the caller (row b belongs to the b-th Byzantine id); only
+ * the kinds that consume them read them.
+ * draws = GENERATED: noise / uniform are ignored; the kernels draw from the library's
+ * counter-based generator, so that only the Byzantine rows move through memory.  A draw is
+ * a pure function of (seed, round, client id, coordinate, stream): Philox4x32-10 with key
+ * (seed mod 2^32, seed div 2^32) and counter (q mod 2^32, q div 2^32, client,
+ * round * 256 + stream) serves the four coordinates 4q..4q+3 (word k mod 4 for coordinate
+ * k).  Stream 0: uniform = (word >> 8) * 2^-24.  Stream 1: a coordinate pair (2p, 2p+1) with
+ * words (a, b) gives u1 = ((a >> 8) + 1) * 2^-24, u2 = (b >> 8) * 2^-24,
+ * radius = sqrt(-2 ln u1), z[2p] = radius cos(2 pi u2), z[2p+1] = radius sin(2 pi u2),
+ * evaluated in float32 (a few ulp from the exactly rounded value).  round < 2^24. */
 typedef struct brace_attack {
   int32_t kind;             /* BRACE_ATTACK_*                                                     */
   float scale;              /* kinds 1, 3                                                         */
@@ -112,6 +128,9 @@ typedef struct brace_attack {
   int64_t noise_ld;
   const float* uniform;     /* device pointer (host pointer for brace_aggregate_host)             */
   int64_t uniform_ld;
+  int32_t draws;            /* BRACE_DRAWS_*                                                      */
+  uint32_t round;           /* GENERATED: round index, < 2^24                                     */
+  uint64_t seed;            /* GENERATED: seed                                                    */
 } brace_attack;
 
 const char* brace_status_string(int status);
@@ -153,9 +172,12 @@ int brace_last_cuda_error(const brace_ctx* ctx);
  * d_honest [n][ld_honest] and writes the f Byzantine rows of d_updates
  * [n][ld_updates]; rows of honest clients are not touched.  d_honest may equal
  * d_updates (in place).  attack->noise / uniform are device pointers.
- * kind NONE or f == 0 does nothing.  Errors: INVALID_ARG (null pointers, ld < d,
- * duplicate or out-of-range ids, missing noise/uniform for a kind that needs
- * them). */
+ * kind NONE or f == 0 does nothing.  The id list is uploaded to the workspace when
+ * it differs from the one already there; that upload is refused while `stream` is
+ * being captured (BRACE_ERR_UNSUPPORTED): call once with a given id list before
+ * capturing.  Errors: INVALID_ARG (null pointers, ld < d, duplicate or
+ * out-of-range ids, missing noise/uniform for a kind that needs them with
+ * draws = SUPPLIED, round >= 2^24 with draws = GENERATED). */
 int brace_inject_attack(brace_ctx* ctx, const brace_attack* attack, const float* d_honest,
                         int64_t ld_honest, float* d_updates, int64_t ld_updates,
                         brace_stream_t stream);
@@ -236,10 +258,23 @@ enum { BRACE_STAT_MEDIAN = 0, BRACE_STAT_TRIMMED_MEAN = 1 };
 int brace_coordinate_stat(brace_ctx* ctx, int32_t kind, int32_t trim, const float* d_updates, int64_t ld,
                           float* d_result, brace_stream_t stream);
 
+/* Rows of the library's own random draws (the generator described at
+ * brace_attack), for inspection and as a building block of synthetic inputs:
+ * row i of d_out [rows][ld] belongs to client first_client + i;
+ *   what = BRACE_DRAW_UNIFORM  d_out[i][k] = the uniform of (seed, round, client, k)
+ *   what = BRACE_DRAW_NORMAL   d_out[i][k] = mu + sigma * z, z the normal of (seed, round, client, k)
+ * Needs no context.  Errors: INVALID_ARG (null, rows < 1, d < 1, ld < d,
+ * first_client < 0, round >= 2^24), CUDA. */
+enum { BRACE_DRAW_UNIFORM = 0, BRACE_DRAW_NORMAL = 1 };
+int brace_draw_matrix(int32_t what, uint64_t seed, uint32_t round, int32_t first_client, int32_t rows, int64_t d,
+                      float* d_out, int64_t ld, float mu, float sigma, brace_stream_t stream);
+
 /* Same round with HOST inputs and outputs: copies h_updates [n][ld] to the
  * caller's device staging matrix d_updates_stage [n][ld], applies `attack`
- * there if attack != NULL (attack->noise / uniform are HOST [f][*_ld] matrices,
- * copied to d_noise_stage / d_uniform_stage of the same shape), aggregates into
+ * there if attack != NULL (with draws = SUPPLIED attack->noise / uniform are HOST
+ * [f][*_ld] matrices, copied to d_noise_stage / d_uniform_stage of the same
+ * shape; with draws = GENERATED nothing but the updates is copied and the two
+ * staging pointers may be NULL), aggregates into
  * d_out_stage [n][out_ld] and copies that to h_out.  All copies are
  * cudaMemcpyAsync on `stream`: pinned host memory makes them asynchronous, and
  * h_out is valid once the stream has been synchronised. */

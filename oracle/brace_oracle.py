@@ -379,6 +379,119 @@ def cost_brace(m, n, d):   # Section 3, Table 1
 
 
 # --------------------------------------------------------------------------
+# Random draws of the attacks that consume randomness (the Gaussian attack the
+# paper names in Section 5.1, and the sparse-noise alteration).  The paper gives
+# no generator; the library draws from a counter-based one so that a draw is a
+# pure function of (seed, round, client, coordinate, stream) and the CPU and GPU
+# sides can each implement it from its published definition: Philox4x32 with 10
+# rounds (Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as
+# 1, 2, 3", SC'11).  This is this module's own implementation of that
+# definition; tests pin it to the known-answer vectors published with it.
+# --------------------------------------------------------------------------
+PHILOX_M0 = 0xD2511F53   # round multipliers
+PHILOX_M1 = 0xCD9E8D57
+PHILOX_W0 = 0x9E3779B9   # key increments per round (golden ratio, sqrt(3) - 1)
+PHILOX_W1 = 0xBB67AE85
+
+STREAM_UNIFORM = 0       # one 32-bit word per coordinate -> uniform in [0, 1)
+STREAM_NORMAL = 1        # two words per coordinate pair -> two standard normals (Box-Muller)
+
+
+def philox4x32_10(counter, key):
+    """The Philox4x32-10 bijection on arrays of counters.
+
+    counter: four uint32 arrays (broadcastable to one shape), key: two uint32
+    values/arrays.  Returns four uint32 arrays.  One round maps
+    (c0, c1, c2, c3), (k0, k1) to
+    (hi(M1*c2) ^ c1 ^ k0, lo(M1*c2), hi(M0*c0) ^ c3 ^ k1, lo(M0*c0));
+    the key advances by (W0, W1) between rounds.
+    """
+    c0, c1, c2, c3 = [np.asarray(c, dtype=np.uint64) for c in counter]
+    k0, k1 = [np.asarray(k, dtype=np.uint64) for k in key]
+    mask = np.uint64(0xFFFFFFFF)
+    for _ in range(10):
+        p0 = np.uint64(PHILOX_M0) * c0          # 32 x 32 -> 64 bits, no overflow in uint64
+        p1 = np.uint64(PHILOX_M1) * c2
+        n0 = (p1 >> np.uint64(32)) ^ c1 ^ k0
+        n1 = p1 & mask
+        n2 = (p0 >> np.uint64(32)) ^ c3 ^ k1
+        n3 = p0 & mask
+        c0, c1, c2, c3 = n0, n1, n2, n3
+        k0 = (k0 + np.uint64(PHILOX_W0)) & mask
+        k1 = (k1 + np.uint64(PHILOX_W1)) & mask
+    return [c.astype(np.uint32) for c in (c0, c1, c2, c3)]
+
+
+def draw_words(seed: int, round_idx: int, client: int, stream: int, d: int, start: int = 0) -> np.ndarray:
+    """The raw 32-bit words of coordinates start .. start + d - 1 (start a multiple
+    of 4) of one client's row of one stream.
+
+    Coordinates are served four at a time: block q = k div 4 is one Philox call
+    with key = (seed mod 2^32, seed div 2^32) and counter
+    (q mod 2^32, q div 2^32, client, round * 256 + stream); word k mod 4 of the
+    result belongs to coordinate k.  round < 2^24, stream < 256.
+    """
+    if not (0 <= seed < 1 << 64 and 0 <= round_idx < 1 << 24 and 0 <= stream < 256 and 0 <= client < 1 << 32):
+        raise ValueError("seed, round, client or stream out of range")
+    if start < 0 or start % 4:
+        raise ValueError("start must be a non-negative multiple of 4")
+    nblk = -(-d // 4)
+    q = np.arange(nblk, dtype=np.uint64) + np.uint64(start // 4)
+    words = philox4x32_10(
+        (q & np.uint64(0xFFFFFFFF), q >> np.uint64(32), np.uint64(client), np.uint64(round_idx * 256 + stream)),
+        (np.uint64(seed & 0xFFFFFFFF), np.uint64(seed >> 32)))
+    return np.stack(words, axis=1).reshape(-1)[:d]
+
+
+def draw_uniform(seed: int, round_idx: int, client: int, d: int, start: int = 0) -> np.ndarray:
+    """float32 [d], uniform on the 2^24 multiples of 2^-24 in [0, 1): the top 24
+    bits of the coordinate's word of STREAM_UNIFORM, times 2^-24 (exact)."""
+    w = draw_words(seed, round_idx, client, STREAM_UNIFORM, d, start)
+    return ((w >> np.uint32(8)).astype(np.float64) * 2.0 ** -24).astype(np.float32)
+
+
+def _cospi_sinpi(x: np.ndarray):
+    """cos(pi x), sin(pi x) for float64 x in [0, 2) with the argument reduced
+    exactly first (x is a multiple of 2^-23 here), so that the zeros of both
+    functions come out as exact zeros."""
+    n = np.rint(2.0 * x)                       # nearest multiple of 1/2
+    r = x - 0.5 * n                            # exact; |r| <= 1/4
+    c, s = np.cos(np.pi * r), np.sin(np.pi * r)
+    quad = n.astype(np.int64) & 3
+    cos_out = np.choose(quad, [c, -s, -c, s])
+    sin_out = np.choose(quad, [s, c, -s, -c])
+    return cos_out, sin_out
+
+
+def draw_normal(seed: int, round_idx: int, client: int, d: int, start: int = 0) -> np.ndarray:
+    """float32 [d] standard normals by the Box-Muller transform, evaluated in
+    float64 and rounded once.  Coordinates 2p and 2p+1 share the words (a, b) of
+    STREAM_NORMAL at those two coordinates: u1 = ((a >> 8) + 1) / 2^24 in (0, 1],
+    u2 = (b >> 8) / 2^24 in [0, 1), radius = sqrt(-2 ln u1);
+    z[2p] = radius * cos(2 pi u2), z[2p+1] = radius * sin(2 pi u2)."""
+    dp = d + (d & 1)
+    w = draw_words(seed, round_idx, client, STREAM_NORMAL, dp, start).reshape(-1, 2)
+    u1 = ((w[:, 0] >> np.uint32(8)).astype(np.float64) + 1.0) * 2.0 ** -24
+    u2 = (w[:, 1] >> np.uint32(8)).astype(np.float64) * 2.0 ** -24
+    radius = np.sqrt(-2.0 * np.log(u1))
+    c, s = _cospi_sinpi(2.0 * u2)
+    z = np.stack([radius * c, radius * s], axis=1).reshape(-1)[:d]
+    return z.astype(np.float32)
+
+
+def attack_draws(kind: int, seed: int, round_idx: int, byz_ids, d: int, start: int = 0):
+    """(noise, uniform) matrices [len(byz_ids), d] an attack of this kind consumes
+    when the library draws for itself: row b holds client byz_ids[b]'s draws for
+    coordinates start .. start + d - 1."""
+    noise = uniform = None
+    if kind in (ATTACK_GAUSSIAN, ATTACK_SPARSE_NOISE):
+        noise = np.stack([draw_normal(seed, round_idx, int(i), d, start) for i in byz_ids])
+    if kind == ATTACK_SPARSE_NOISE:
+        uniform = np.stack([draw_uniform(seed, round_idx, int(i), d, start) for i in byz_ids])
+    return noise, uniform
+
+
+# --------------------------------------------------------------------------
 # Section 3 (threat model): Byzantine clients alter their vectors before the
 # ring starts.  The five synthetic alterations of the benchmark workloads.
 # --------------------------------------------------------------------------

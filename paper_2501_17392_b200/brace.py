@@ -20,6 +20,8 @@ RULE_SIGN_CONSENSUS, RULE_SUM, RULE_MAJORITY_SIGN, RULE_ABS_CONSENSUS = 0, 1, 2,
 AGG_AUTO, AGG_STEPWISE, AGG_FUSED = 0, 1, 2
 STAT_MEDIAN, STAT_TRIMMED_MEAN = 0, 1
 ATTACK_NONE, ATTACK_SCALE_OWN, ATTACK_GAUSSIAN, ATTACK_SCALED_MEAN, ATTACK_MEAN_SHIFT, ATTACK_SPARSE_NOISE = range(6)
+DRAWS_SUPPLIED, DRAWS_GENERATED = 0, 1
+DRAW_UNIFORM, DRAW_NORMAL = 0, 1
 
 
 class Params(C.Structure):
@@ -30,7 +32,8 @@ class Params(C.Structure):
 class Attack(C.Structure):
     _fields_ = [("kind", C.c_int32), ("scale", C.c_float), ("sigma", C.c_float), ("kappa", C.c_float),
                 ("prob", C.c_float), ("h_byz_ids", C.POINTER(C.c_int32)), ("noise", C.c_void_p),
-                ("noise_ld", C.c_int64), ("uniform", C.c_void_p), ("uniform_ld", C.c_int64)]
+                ("noise_ld", C.c_int64), ("uniform", C.c_void_p), ("uniform_ld", C.c_int64),
+                ("draws", C.c_int32), ("round", C.c_uint32), ("seed", C.c_uint64)]
 
 
 class Cost(C.Structure):
@@ -61,6 +64,8 @@ SIGNATURES = {
     "brace_comm_cost": (C.c_int, [C.c_void_p, C.c_int32, C.POINTER(Cost)]),
     "brace_inject_attack": (C.c_int, [C.c_void_p, C.POINTER(Attack), C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
                                       C.c_void_p]),
+    "brace_draw_matrix": (C.c_int, [C.c_int32, C.c_uint64, C.c_uint32, C.c_int32, C.c_int32, C.c_int64, C.c_void_p,
+                                    C.c_int64, C.c_float, C.c_float, C.c_void_p]),
     "brace_quantize": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p]),
     "brace_ring_reduce_scatter_step": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p]),
     "brace_consensus": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
@@ -131,10 +136,14 @@ def _ptr(t) -> int:
 
 
 def make_attack(kind: int, *, scale=1.0, sigma=1.0, kappa=3.0, prob=0.1, byz_ids=None, noise=None,
-                uniform=None) -> Attack:
-    """Build the attack descriptor; keeps the id array alive on the returned object."""
+                uniform=None, seed=None, round_idx=0) -> Attack:
+    """Build the attack descriptor; keeps the id array alive on the returned object.
+    With `seed` given the library draws the attack's random numbers itself from
+    (seed, round_idx); otherwise `noise` / `uniform` supply them."""
     a = Attack()
     a.kind, a.scale, a.sigma, a.kappa, a.prob = kind, scale, sigma, kappa, prob
+    if seed is not None:
+        a.draws, a.seed, a.round = DRAWS_GENERATED, int(seed), int(round_idx)
     if byz_ids is not None:
         arr = (C.c_int32 * len(byz_ids))(*[int(i) for i in byz_ids])
         a._ids_keepalive = arr
@@ -146,6 +155,19 @@ def make_attack(kind: int, *, scale=1.0, sigma=1.0, kappa=3.0, prob=0.1, byz_ids
         a._uniform_keepalive = uniform
         a.uniform, a.uniform_ld = _ptr(uniform), uniform.stride(0)
     return a
+
+
+def draw_matrix_status(what: int, seed: int, round_idx: int, first_client: int, out: torch.Tensor, d: int,
+                       mu=0.0, sigma=1.0, stream=None) -> int:
+    return lib().brace_draw_matrix(what, seed, round_idx, first_client, out.shape[0], d, _ptr(out), out.stride(0),
+                                   float(mu), float(sigma), _stream(stream))
+
+
+def draw_matrix(what: int, seed: int, round_idx: int, first_client: int, out: torch.Tensor, d: int, mu=0.0,
+                sigma=1.0, stream=None):
+    """Fill `out` [rows, ld] with the library's own uniform / normal draws of clients
+    first_client .. first_client + rows - 1 (the draws attacks 2 and 5 consume)."""
+    _check(draw_matrix_status(what, seed, round_idx, first_client, out, d, mu, sigma, stream), "brace_draw_matrix")
 
 
 def aggregate_static_status(n: int, d: int, params: Params, updates: torch.Tensor, out: torch.Tensor,

@@ -19,7 +19,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int64_t kMailAlign = 128;   // mailbox length granularity (entries)
-constexpr int kSmCount = 148;
+constexpr int kDefaultSmCount = 148;  // B200; replaced by the device's own count when a context gets a workspace
 
 enum Phase { kIdle = 0, kReducing = 1, kReduced = 2, kConsensusDone = 3, kGathering = 4, kDone = 5 };
 
@@ -46,15 +46,21 @@ struct brace_ctx {
   int rs_done = 0;   // share-reduce hops completed in the current round
   int ag_done = 0;   // share-only hops completed in the current round
   int last_cuda = 0;
+  bool no_ctx_call = false;   // the context lives on the stack of a context-free entry point
   // ids currently stored in d_ids (Byzantine first, then honest), and their staging copy
   std::vector<int> ids_on_device;
   std::vector<int> ids_staging;
+  std::vector<char> is_byz;
+  bool ids_valid = false;
+  int sm_count = kDefaultSmCount;
+  size_t stats_smem_set[3] = {0, 0, 0};   // dynamic shared memory already granted to the staged statistics kernels
   // launch tuning (0 = default)
   int fused_variant = 0;
   int fused_grid = 0;
   int step_vpt = 0;
   int spread_mode = 0;   // 0/1 = owner row + share-only launch when the layout allows, 2 = fused kernel writes all rows
   int stats_vw = 0;
+  int stats_table = 0;   // 1 = statistics kernel addresses rows through the offset table even when they are consecutive
 };
 
 namespace {
@@ -127,13 +133,18 @@ void consensus_thresholds(const brace_params* p, int n, int* hi, int* lo) {
   }
 }
 
+// cudaError_t of the last failed runtime call made by a context-free entry point on this thread
+thread_local int g_last_cuda_no_ctx = 0;
+
 int cuda_fail(brace_ctx* ctx, cudaError_t err) {
   ctx->last_cuda = (int)err;
+  if (ctx->no_ctx_call) g_last_cuda_no_ctx = (int)err;
   return BRACE_ERR_CUDA;
 }
 
-int check_launch(brace_ctx* ctx) {
+int check_launch(brace_ctx* ctx, cudaError_t launch_err = cudaSuccess) {
   cudaError_t err = cudaGetLastError();
+  if (launch_err != cudaSuccess) err = launch_err;
   if (err != cudaSuccess) return cuda_fail(ctx, err);
   return BRACE_OK;
 }
@@ -148,7 +159,7 @@ inline unsigned tiles(int64_t items, int64_t per_block) {
 // Launch with programmatic stream serialization: the kernel may begin while its
 // predecessor on the stream drains; it synchronises on the device (pdl_wait).
 template <typename... KArgs, typename... Args>
-void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -159,7 +170,7 @@ void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 bool vec_layout_ok(const brace_ctx* ctx, const float* U, int64_t ld) {
@@ -167,6 +178,7 @@ bool vec_layout_ok(const brace_ctx* ctx, const float* U, int64_t ld) {
 }
 
 int launch_rs_step(brace_ctx* ctx, int step, const float* U, int64_t ld, cudaStream_t st) {
+  cudaError_t perr = cudaSuccess;
   const int n = ctx->n;
   const int in_set = step & 1, out_set = (step + 1) & 1;
   const bool vec = vec_layout_ok(ctx, U, ld);
@@ -174,14 +186,14 @@ int launch_rs_step(brace_ctx* ctx, int step, const float* U, int64_t ld, cudaStr
   int vpt = 0;
   if (vec) {
     vpt = ctx->step_vpt > 0 ? ctx->step_vpt : 4;
-    while (vpt > 1 && (int64_t)n * ((ctx->seg_max + 1024 * vpt - 1) / (1024 * vpt)) < 4 * kSmCount) vpt >>= 1;
+    while (vpt > 1 && (int64_t)n * ((ctx->seg_max + 1024 * vpt - 1) / (1024 * vpt)) < 4 * ctx->sm_count) vpt >>= 1;
   }
   const int64_t per_block = vec ? (int64_t)kThreads * 4 * vpt : kThreads;
   dim3 grid(tiles(ctx->seg_max, per_block), (unsigned)n);
   const bool zs = ctx->p.zero_sign != 0;
   const int zsv = ctx->p.zero_sign;
 #define BRACE_RS_SIGN(P, VPT, ZS)                                                                            \
-  launch_pdl(rs_step_sign_kernel<P, VPT, ZS>, grid, dim3(kThreads), st, ctx->pt, U, ld,                       \
+  perr = launch_pdl(rs_step_sign_kernel<P, VPT, ZS>, grid, dim3(kThreads), st, ctx->pt, U, ld,                       \
              (const P*)ctx->mail[in_set], (P*)ctx->mail[out_set], ctx->seg_pad, step, zsv)
 #define BRACE_RS_SIGN_P(P)                                                                         \
   do {                                                                                             \
@@ -195,10 +207,10 @@ int launch_rs_step(brace_ctx* ctx, int step, const float* U, int64_t ld, cudaStr
   if (ctx->p.rule == BRACE_RULE_SUM) {
     dim3 gsum(tiles(ctx->seg_max, vec ? kThreads * 4 : kThreads), (unsigned)n);
     if (vec)
-      launch_pdl(rs_step_sum_kernel<true>, gsum, dim3(kThreads), st, ctx->pt, U, ld,
+      perr = launch_pdl(rs_step_sum_kernel<true>, gsum, dim3(kThreads), st, ctx->pt, U, ld,
                  (const float*)ctx->mail[in_set], (float*)ctx->mail[out_set], ctx->seg_pad, step);
     else
-      launch_pdl(rs_step_sum_kernel<false>, gsum, dim3(kThreads), st, ctx->pt, U, ld,
+      perr = launch_pdl(rs_step_sum_kernel<false>, gsum, dim3(kThreads), st, ctx->pt, U, ld,
                  (const float*)ctx->mail[in_set], (float*)ctx->mail[out_set], ctx->seg_pad, step);
   } else if (ctx->entry_bytes == 1) {
     BRACE_RS_SIGN_P(int8_t);
@@ -207,53 +219,55 @@ int launch_rs_step(brace_ctx* ctx, int step, const float* U, int64_t ld, cudaStr
   }
 #undef BRACE_RS_SIGN_P
 #undef BRACE_RS_SIGN
-  return check_launch(ctx);
+  return check_launch(ctx, perr);
 }
 
 int launch_consensus(brace_ctx* ctx, void* out, int64_t out_ld, cudaStream_t st) {
+  cudaError_t perr = cudaSuccess;
   const int n = ctx->n;
   const int set = (n - 1) & 1;   // the last hop n-2 wrote set (n-1)&1
   if (ctx->p.rule == BRACE_RULE_SUM) {
     const bool vec = (ctx->p.granule % 4 == 0) && (out_ld % 4 == 0) && aligned16(out);
     dim3 grid(tiles(ctx->seg_max, vec ? kThreads * 4 : kThreads), (unsigned)n);
     if (vec)
-      launch_pdl(consensus_sum_kernel<true>, grid, dim3(kThreads), st, ctx->pt, (const float*)ctx->mail[set],
+      perr = launch_pdl(consensus_sum_kernel<true>, grid, dim3(kThreads), st, ctx->pt, (const float*)ctx->mail[set],
                  ctx->seg_pad, (float*)out, out_ld, ctx->p.mean);
     else
-      launch_pdl(consensus_sum_kernel<false>, grid, dim3(kThreads), st, ctx->pt, (const float*)ctx->mail[set],
+      perr = launch_pdl(consensus_sum_kernel<false>, grid, dim3(kThreads), st, ctx->pt, (const float*)ctx->mail[set],
                  ctx->seg_pad, (float*)out, out_ld, ctx->p.mean);
   } else {
     dim3 grid(tiles(ctx->seg_max / 32 + 2, kThreads), (unsigned)n);
     if (ctx->entry_bytes == 1)
-      launch_pdl(consensus_sign_kernel<int8_t>, grid, dim3(kThreads), st, ctx->pt, (const int8_t*)ctx->mail[set],
+      perr = launch_pdl(consensus_sign_kernel<int8_t>, grid, dim3(kThreads), st, ctx->pt, (const int8_t*)ctx->mail[set],
                  ctx->seg_pad, (uint32_t*)out, out_ld, ctx->lam_i, ctx->lam_lo);
     else
-      launch_pdl(consensus_sign_kernel<int16_t>, grid, dim3(kThreads), st, ctx->pt, (const int16_t*)ctx->mail[set],
+      perr = launch_pdl(consensus_sign_kernel<int16_t>, grid, dim3(kThreads), st, ctx->pt, (const int16_t*)ctx->mail[set],
                  ctx->seg_pad, (uint32_t*)out, out_ld, ctx->lam_i, ctx->lam_lo);
   }
-  return check_launch(ctx);
+  return check_launch(ctx, perr);
 }
 
 int launch_ag_step(brace_ctx* ctx, int step, void* out, int64_t out_ld, cudaStream_t st) {
+  cudaError_t perr = cudaSuccess;
   const int n = ctx->n;
   if (ctx->p.rule == BRACE_RULE_SUM) {
     const bool vec = (ctx->p.granule % 4 == 0) && (out_ld % 4 == 0) && aligned16(out);
     dim3 grid(tiles(ctx->seg_max, vec ? kThreads * 4 : kThreads), (unsigned)n);
     if (vec)
-      launch_pdl(ag_step_f32_kernel<true>, grid, dim3(kThreads), st, ctx->pt, (float*)out, out_ld, step);
+      perr = launch_pdl(ag_step_f32_kernel<true>, grid, dim3(kThreads), st, ctx->pt, (float*)out, out_ld, step);
     else
-      launch_pdl(ag_step_f32_kernel<false>, grid, dim3(kThreads), st, ctx->pt, (float*)out, out_ld, step);
+      perr = launch_pdl(ag_step_f32_kernel<false>, grid, dim3(kThreads), st, ctx->pt, (float*)out, out_ld, step);
   } else {
     const bool wide = (ctx->p.granule % 128 == 0) && (out_ld % 4 == 0) && aligned16(out);
     if (wide) {
       dim3 grid(tiles(ctx->seg_max / 128 + 2, kThreads), (unsigned)n);
-      launch_pdl(ag_step_bits_kernel<4>, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, step);
+      perr = launch_pdl(ag_step_bits_kernel<4>, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, step);
     } else {
       dim3 grid(tiles(ctx->seg_max / 32 + 2, kThreads), (unsigned)n);
-      launch_pdl(ag_step_bits_kernel<1>, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, step);
+      perr = launch_pdl(ag_step_bits_kernel<1>, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, step);
     }
   }
-  return check_launch(ctx);
+  return check_launch(ctx, perr);
 }
 
 // ---- fused round ------------------------------------------------------------------------
@@ -264,9 +278,7 @@ bool fused_layout_ok(const brace_ctx* ctx, const float* U, int64_t ld, const voi
   return true;
 }
 
-template <int VPT>
-void fused_geometry(const brace_ctx* ctx, FusedArgs& a) {
-  const int64_t tile = 256 * 4 * VPT;
+void fused_geometry(const brace_ctx* ctx, FusedArgs& a, int64_t tile) {
   a.tiles_per_seg = (int)((ctx->seg_max + tile - 1) / tile);
   if (a.tiles_per_seg < 1) a.tiles_per_seg = 1;
   a.units = (int64_t)a.tiles_per_seg * ctx->n;
@@ -299,25 +311,25 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
   auto grid_for = [&](int64_t units) -> unsigned {
     int64_t g = units;
     if (ctx->fused_grid > 0 && g > ctx->fused_grid) g = ctx->fused_grid;
-    const int64_t cap = (int64_t)kSmCount * 4096;
+    const int64_t cap = (int64_t)ctx->sm_count * 4096;
     if (g > cap) g = cap;
     return (unsigned)(g > 0 ? g : 1);
   };
-#define BRACE_FUSED_SIGN(VPT, UNR)                                                              \
+#define BRACE_FUSED_SIGN(VPT, UNR, TPB)                                                         \
   do {                                                                                          \
-    fused_geometry<VPT>(ctx, a);                                                                \
+    fused_geometry(ctx, a, (int64_t)TPB * 4 * VPT);                                             \
     const unsigned g = grid_for(a.units);                                                       \
     if (ctx->entry_bytes == 1) {                                                                \
-      if (zs) fused_sign_kernel<int8_t, VPT, UNR, true><<<g, 256, 0, st>>>(a);                  \
-      else    fused_sign_kernel<int8_t, VPT, UNR, false><<<g, 256, 0, st>>>(a);                 \
+      if (zs) fused_sign_kernel<int8_t, VPT, UNR, true, TPB><<<g, TPB, 0, st>>>(a);             \
+      else    fused_sign_kernel<int8_t, VPT, UNR, false, TPB><<<g, TPB, 0, st>>>(a);            \
     } else {                                                                                    \
-      if (zs) fused_sign_kernel<int16_t, VPT, UNR, true><<<g, 256, 0, st>>>(a);                 \
-      else    fused_sign_kernel<int16_t, VPT, UNR, false><<<g, 256, 0, st>>>(a);                \
+      if (zs) fused_sign_kernel<int16_t, VPT, UNR, true, TPB><<<g, TPB, 0, st>>>(a);            \
+      else    fused_sign_kernel<int16_t, VPT, UNR, false, TPB><<<g, TPB, 0, st>>>(a);           \
     }                                                                                           \
   } while (0)
 #define BRACE_FUSED_SUM(VPT, UNR)                                                               \
   do {                                                                                          \
-    fused_geometry<VPT>(ctx, a);                                                                \
+    fused_geometry(ctx, a, (int64_t)256 * 4 * VPT);                                             \
     const unsigned g = grid_for(a.units);                                                       \
     fused_sum_kernel<VPT, UNR><<<g, 256, 0, st>>>(a);                                           \
   } while (0)
@@ -329,11 +341,15 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
     }
   } else {
     switch (variant) {
-      case 2: BRACE_FUSED_SIGN(2, 4); break;
-      case 3: BRACE_FUSED_SIGN(1, 4); break;
-      case 4: BRACE_FUSED_SIGN(2, 8); break;
-      case 5: BRACE_FUSED_SIGN(1, 16); break;
-      default: BRACE_FUSED_SIGN(1, 8); break;
+      case 2: BRACE_FUSED_SIGN(2, 4, 256); break;
+      case 3: BRACE_FUSED_SIGN(1, 4, 256); break;
+      case 4: BRACE_FUSED_SIGN(2, 8, 256); break;
+      case 5: BRACE_FUSED_SIGN(1, 16, 256); break;
+      case 6: BRACE_FUSED_SIGN(1, 24, 256); break;
+      case 7: BRACE_FUSED_SIGN(1, 8, 128); break;
+      case 8: BRACE_FUSED_SIGN(1, 16, 128); break;
+      case 9: BRACE_FUSED_SIGN(1, 24, 128); break;
+      default: BRACE_FUSED_SIGN(1, 8, 256); break;
     }
   }
 #undef BRACE_FUSED_SIGN
@@ -343,8 +359,9 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
   const int rows_per_group = 8;
   dim3 grid(tiles(ctx->seg_max / 128 + 2, kThreads), (unsigned)ctx->n,
             (unsigned)((ctx->n + rows_per_group - 1) / rows_per_group));
-  launch_pdl(ag_all_bits_kernel, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, rows_per_group);
-  return check_launch(ctx);
+  const cudaError_t perr =
+      launch_pdl(ag_all_bits_kernel, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, rows_per_group);
+  return check_launch(ctx, perr);
 }
 
 // ---- argument checks shared by the ring calls -----------------------------------------------
@@ -389,9 +406,9 @@ int run_stepwise(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
 // device copy is already current, so steady-state calls enqueue kernels only.
 int stage_ids(brace_ctx* ctx, const int32_t* h_byz_ids, cudaStream_t st) {
   const int n = ctx->n, f = ctx->f;
-  std::vector<int>& ids = ctx->ids_staging;
-  ids.assign((size_t)n, 0);
-  std::vector<char> is_byz((size_t)n, 0);
+  std::vector<int>& ids = ctx->ids_staging;          // sized n at init: nothing is allocated here
+  std::vector<char>& is_byz = ctx->is_byz;
+  std::fill(is_byz.begin(), is_byz.end(), (char)0);
   for (int b = 0; b < f; ++b) {
     const int id = h_byz_ids ? h_byz_ids[b] : b;
     if (id < 0 || id >= n || is_byz[(size_t)id]) return BRACE_ERR_INVALID_ARG;
@@ -401,10 +418,17 @@ int stage_ids(brace_ctx* ctx, const int32_t* h_byz_ids, cudaStream_t st) {
   int pos = f;
   for (int i = 0; i < n; ++i)
     if (!is_byz[(size_t)i]) ids[(size_t)pos++] = i;
-  if (ids == ctx->ids_on_device) return BRACE_OK;
-  cudaError_t err = cudaMemcpyAsync(ctx->d_ids, ids.data(), (size_t)n * sizeof(int), cudaMemcpyHostToDevice, st);
+  if (ctx->ids_valid && ids == ctx->ids_on_device) return BRACE_OK;
+  // a new id list has to be uploaded: not while the stream is being captured (the copy would be
+  // recorded instead of executed, and later calls would skip it)
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  cudaError_t err = cudaStreamIsCapturing(st, &cap);
   if (err != cudaSuccess) return cuda_fail(ctx, err);
-  ctx->ids_on_device = ids;
+  if (cap != cudaStreamCaptureStatusNone) return BRACE_ERR_UNSUPPORTED;
+  err = cudaMemcpyAsync(ctx->d_ids, ids.data(), (size_t)n * sizeof(int), cudaMemcpyHostToDevice, st);
+  if (err != cudaSuccess) return cuda_fail(ctx, err);
+  ctx->ids_on_device = ids;                           // same size: no allocation
+  ctx->ids_valid = true;
   return BRACE_OK;
 }
 
@@ -416,24 +440,61 @@ int inject_impl(brace_ctx* ctx, const brace_attack* atk, const float* H, int64_t
   if (!H || !Uo || ld_h < ctx->d || ld_u < ctx->d) return BRACE_ERR_INVALID_ARG;
   const int kind = atk->kind;
   const bool needs_noise = kind == BRACE_ATTACK_GAUSSIAN || kind == BRACE_ATTACK_SPARSE_NOISE;
-  if (needs_noise && (!atk->noise || atk->noise_ld < ctx->d)) return BRACE_ERR_INVALID_ARG;
-  if (kind == BRACE_ATTACK_SPARSE_NOISE && (!atk->uniform || atk->uniform_ld < ctx->d)) return BRACE_ERR_INVALID_ARG;
+  if (atk->draws != BRACE_DRAWS_SUPPLIED && atk->draws != BRACE_DRAWS_GENERATED) return BRACE_ERR_INVALID_ARG;
+  const bool generated = needs_noise && atk->draws == BRACE_DRAWS_GENERATED;
+  if (generated && atk->round >= (1u << 24)) return BRACE_ERR_INVALID_ARG;
+  if (needs_noise && !generated && (!atk->noise || atk->noise_ld < ctx->d)) return BRACE_ERR_INVALID_ARG;
+  if (kind == BRACE_ATTACK_SPARSE_NOISE && !generated && (!atk->uniform || atk->uniform_ld < ctx->d))
+    return BRACE_ERR_INVALID_ARG;
   int rc = stage_ids(ctx, atk->h_byz_ids, st);
   if (rc != BRACE_OK) return rc;
   const bool rows16 = (ld_h % 4 == 0) && (ld_u % 4 == 0) && aligned16(H) && aligned16(Uo);
+  if (generated) {
+    dim3 grid(tiles((ctx->d + 3) / 4, kThreads), (unsigned)ctx->f);
+    inject_generated_kernel<<<grid, kThreads, 0, st>>>(kind, ctx->d_ids, Uo, ld_u, ctx->d, atk->seed, atk->round,
+                                                      atk->sigma, atk->prob, (ld_u % 4 == 0 && aligned16(Uo)) ? 1 : 0);
+    return check_launch(ctx);
+  }
   if (kind == BRACE_ATTACK_SCALED_MEAN || kind == BRACE_ATTACK_MEAN_SHIFT) {
     const int m = ctx->n - ctx->f;
     const int mpad = (m + 7) / 8 * 8;
     if (kind == BRACE_ATTACK_MEAN_SHIFT && m <= 127 && ctx->stats_vw == 0) {
       // two passes: register-resident variant, one coordinate per thread, all honest values in registers
+      const std::vector<int>& ids = ctx->ids_on_device;
+      const int f = ctx->f;
+      bool strided = (ld_h * 4 < ((int64_t)1 << 32)) && ctx->stats_table == 0;
+      for (int r = 1; r < m && strided; ++r) strided = ids[(size_t)f + r] == ids[(size_t)f] + r;
+      for (int b = 1; b < f && strided; ++b) strided = ids[(size_t)b] == ids[0] + b;
+      const unsigned blocks = tiles(ctx->d, 128);
+      if (strided) {
+        const float* H0 = H + (int64_t)ids[(size_t)f] * ld_h;
+        float* U0 = Uo + (int64_t)ids[0] * ld_u;
+        HonestRows none{};
+#define BRACE_STATS_REG(MFULL)                                                                               \
+  case MFULL:                                                                                                \
+    inject_stats_reg_kernel<MFULL, 3, true><<<blocks, 128, 0, st>>>(kind, none, (uint32_t)(ld_h * 4), nullptr, f, m, \
+                                                                    H0, U0, ld_u, ctx->d, atk->scale, atk->kappa);    \
+    break
+        switch (m / 4 * 4) {
+          BRACE_STATS_REG(0); BRACE_STATS_REG(4); BRACE_STATS_REG(8); BRACE_STATS_REG(12); BRACE_STATS_REG(16);
+          BRACE_STATS_REG(20); BRACE_STATS_REG(24); BRACE_STATS_REG(28); BRACE_STATS_REG(32); BRACE_STATS_REG(36);
+          BRACE_STATS_REG(40); BRACE_STATS_REG(44); BRACE_STATS_REG(48); BRACE_STATS_REG(52); BRACE_STATS_REG(56);
+          BRACE_STATS_REG(60); BRACE_STATS_REG(64); BRACE_STATS_REG(68); BRACE_STATS_REG(72); BRACE_STATS_REG(76);
+          BRACE_STATS_REG(80); BRACE_STATS_REG(84); BRACE_STATS_REG(88); BRACE_STATS_REG(92); BRACE_STATS_REG(96);
+          BRACE_STATS_REG(100); BRACE_STATS_REG(104); BRACE_STATS_REG(108); BRACE_STATS_REG(112);
+          BRACE_STATS_REG(116); BRACE_STATS_REG(120);
+          default: BRACE_STATS_REG(124);
+        }
+#undef BRACE_STATS_REG
+        return check_launch(ctx);
+      }
       HonestRows rows;
       for (int r = 0; r < 128; ++r)
-        rows.byte_off[r] = (int64_t)ctx->ids_on_device[(size_t)ctx->f + (size_t)(r < m ? r : m - 1)] * ld_h * 4;
-      const unsigned blocks = tiles(ctx->d, 128);
-#define BRACE_STATS_REG(MFULL)                                                                          \
-  case MFULL:                                                                                           \
-    inject_stats_reg_kernel<MFULL><<<blocks, 128, 0, st>>>(kind, rows, ctx->d_ids, ctx->f, m, H, Uo, ld_u, \
-                                                           ctx->d, atk->scale, atk->kappa);             \
+        rows.byte_off[r] = (int64_t)ids[(size_t)f + (size_t)(r < m ? r : m - 1)] * ld_h * 4;
+#define BRACE_STATS_REG(MFULL)                                                                                \
+  case MFULL:                                                                                                 \
+    inject_stats_reg_kernel<MFULL, 7, false><<<blocks, 128, 0, st>>>(kind, rows, 0u, ctx->d_ids, f, m, H, Uo, ld_u, \
+                                                                     ctx->d, atk->scale, atk->kappa);         \
     break
       switch (m / 8 * 8) {
         BRACE_STATS_REG(0); BRACE_STATS_REG(8); BRACE_STATS_REG(16); BRACE_STATS_REG(24); BRACE_STATS_REG(32);
@@ -457,12 +518,14 @@ int inject_impl(brace_ctx* ctx, const brace_attack* atk, const float* H, int64_t
     if (layout_ok && smem <= 200 * 1024) {
       auto kern = vw == 1 ? inject_stats_smem_kernel<1, 12>
                           : (vw == 2 ? inject_stats_smem_kernel<2, 12> : inject_stats_smem_kernel<4, 12>);
-      if (smem > 48 * 1024) {
+      size_t& granted = ctx->stats_smem_set[vw == 1 ? 0 : (vw == 2 ? 1 : 2)];
+      if (smem > 48 * 1024 && smem > granted) {      // once per context and kernel, not on every call
         cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return cuda_fail(ctx, err);
+        granted = smem;
       }
       int64_t blocks = (ctx->d + (int64_t)T * vw - 1) / ((int64_t)T * vw);
-      const int64_t cap = (int64_t)kSmCount * 64;
+      const int64_t cap = (int64_t)ctx->sm_count * 64;
       if (blocks > cap) blocks = cap;
       kern<<<(unsigned)blocks, T, smem, st>>>(kind, ctx->d_ids, ctx->f, ctx->n, H, ld_h, Uo, ld_u, ctx->d,
                                              atk->scale, atk->kappa);
@@ -470,7 +533,7 @@ int inject_impl(brace_ctx* ctx, const brace_attack* atk, const float* H, int64_t
       // two passes over the honest rows in global memory: keep the set of coordinates in
       // flight small enough that the second pass finds the first one's lines in L2
       int64_t blocks = (ctx->d + kThreads - 1) / kThreads;
-      const int64_t cap = (int64_t)kSmCount * 4;
+      const int64_t cap = (int64_t)ctx->sm_count * 4;
       if (blocks > cap) blocks = cap;
       inject_stats_kernel<8><<<(unsigned)blocks, kThreads, 0, st>>>(kind, ctx->d_ids, ctx->f, ctx->n, H, ld_h, Uo,
                                                                    ld_u, ctx->d, atk->scale, atk->kappa);
@@ -519,36 +582,12 @@ int aggregate_impl(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_
 // ---- round without a caller workspace ---------------------------------------------------------
 // Mailbox scratch for brace_aggregate_static.  Every GPU that loads the library
 // holds these bytes until the process exits.  In host code the symbol's name is
-// only a handle: the device address is fetched once per device with
-// cudaGetSymbolAddress and that pointer is what the kernels receive.
+// only a handle: the device address is fetched with cudaGetSymbolAddress (on
+// every call, for the device that is current then: the lookup allocates nothing,
+// and a cached pointer would go stale after cudaDeviceReset or under another
+// context) and that pointer is what the kernels receive.
 constexpr size_t kStaticScratchBytes = (size_t)BRACE_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
-
-namespace {
-
-constexpr int kMaxDevices = 64;
-std::mutex g_static_mutex;
-void* g_static_ptr[kMaxDevices] = {nullptr};
-
-// Device address of g_static_scratch on the current device (looked up on first use).
-cudaError_t static_scratch_for_current_device(void** out) {
-  int dev = -1;
-  cudaError_t err = cudaGetDevice(&dev);
-  if (err != cudaSuccess) return err;
-  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  std::lock_guard<std::mutex> lock(g_static_mutex);
-  if (!g_static_ptr[dev]) {
-    void* ptr = nullptr;
-    err = cudaGetSymbolAddress(&ptr, g_static_scratch);
-    if (err != cudaSuccess) return err;
-    if (!ptr || (reinterpret_cast<uintptr_t>(ptr) & 255u) != 0) return cudaErrorInvalidSymbol;
-    g_static_ptr[dev] = ptr;
-  }
-  *out = g_static_ptr[dev];
-  return cudaSuccess;
-}
-
-}  // namespace
 
 // =============================================================================================
 // C ABI
@@ -599,6 +638,14 @@ int brace_init(brace_ctx** out, int32_t n, int32_t f, int64_t d, const brace_par
   }
   brace_ctx* ctx = new (std::nothrow) brace_ctx();
   if (!ctx) return BRACE_ERR_INVALID_ARG;
+  try {                                              // host vectors are sized once, here
+    ctx->ids_on_device.assign((size_t)n, 0);
+    ctx->ids_staging.assign((size_t)n, 0);
+    ctx->is_byz.assign((size_t)n, 0);
+  } catch (...) {
+    delete ctx;
+    return BRACE_ERR_INVALID_ARG;
+  }
   ctx->n = n;
   ctx->f = f;
   ctx->d = d;
@@ -615,6 +662,10 @@ int brace_init(brace_ctx** out, int32_t n, int32_t f, int64_t d, const brace_par
     ctx->mail[0] = ctx->ws;
     ctx->mail[1] = ctx->ws + one_set;
     ctx->d_ids = reinterpret_cast<int*>(ctx->ws + 2 * one_set);
+    int dev = 0, sms = 0;                            // grid sizing follows the device that is current now
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      ctx->sm_count = sms;
   }
   *out = ctx;
   return BRACE_OK;
@@ -661,7 +712,7 @@ int brace_comm_cost(const brace_ctx* ctx, int32_t m_bits, brace_cost* cost) {
   return BRACE_OK;
 }
 
-int brace_last_cuda_error(const brace_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+int brace_last_cuda_error(const brace_ctx* ctx) { return ctx ? ctx->last_cuda : g_last_cuda_no_ctx; }
 
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid) {
   if (!ctx || fused_variant < 0 || fused_grid < 0) return BRACE_ERR_INVALID_ARG;
@@ -670,13 +721,14 @@ int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid) 
   const int stats_code = fused_variant / 100;    // hundreds digit: floats per thread of the statistics kernel
   const int step_code = (fused_variant / 10) % 10;   // tens digit: float4 per thread of the hop kernel
   fused_variant %= 10;
-  if (fused_variant > 5 || (step_code != 0 && step_code != 1 && step_code != 2 && step_code != 4) ||
-      (stats_code != 0 && stats_code != 1 && stats_code != 2 && stats_code != 4))
+  if (fused_variant > 9 || (step_code != 0 && step_code != 1 && step_code != 2 && step_code != 4) ||
+      (stats_code != 0 && stats_code != 1 && stats_code != 2 && stats_code != 4 && stats_code != 8))
     return BRACE_ERR_INVALID_ARG;
   if (spread_code < 0 || spread_code > 2) return BRACE_ERR_INVALID_ARG;
   ctx->spread_mode = spread_code;
   ctx->step_vpt = step_code;
-  ctx->stats_vw = stats_code;
+  ctx->stats_vw = stats_code == 8 ? 0 : stats_code;
+  ctx->stats_table = stats_code == 8 ? 1 : 0;
   ctx->fused_variant = fused_variant;
   ctx->fused_grid = fused_grid;
   return BRACE_OK;
@@ -687,6 +739,20 @@ int brace_inject_attack(brace_ctx* ctx, const brace_attack* attack, const float*
   int rc = check_device_ctx(ctx);
   if (rc != BRACE_OK) return rc;
   return inject_impl(ctx, attack, d_honest, ld_honest, d_updates, ld_updates, static_cast<cudaStream_t>(stream));
+}
+
+int brace_draw_matrix(int32_t what, uint64_t seed, uint32_t round, int32_t first_client, int32_t rows, int64_t d,
+                      float* d_out, int64_t ld, float mu, float sigma, brace_stream_t stream) {
+  if ((what != BRACE_DRAW_UNIFORM && what != BRACE_DRAW_NORMAL) || !d_out || rows < 1 || d < 1 || ld < d ||
+      first_client < 0 || round >= (1u << 24) || rows > 65535)
+    return BRACE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_out) & 3u) != 0) return BRACE_ERR_INVALID_ARG;
+  brace_ctx ctx;
+  ctx.no_ctx_call = true;
+  dim3 grid(tiles((d + 3) / 4, kThreads), (unsigned)rows);
+  draw_matrix_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      what, seed, round, first_client, d_out, ld, d, mu, sigma, (ld % 4 == 0 && aligned16(d_out)) ? 1 : 0);
+  return check_launch(&ctx);
 }
 
 int brace_quantize(brace_ctx* ctx, const float* d_updates, int64_t ld, int8_t* d_q, int64_t ld_q,
@@ -835,8 +901,10 @@ int brace_aggregate_host(brace_ctx* ctx, const brace_attack* attack, const float
   const bool do_attack = attack && attack->kind != BRACE_ATTACK_NONE && f > 0;
   if (do_attack) {
     dev_attack = *attack;
-    const bool needs_noise = attack->kind == BRACE_ATTACK_GAUSSIAN || attack->kind == BRACE_ATTACK_SPARSE_NOISE;
-    const bool needs_unif = attack->kind == BRACE_ATTACK_SPARSE_NOISE;
+    const bool supplied = attack->draws == BRACE_DRAWS_SUPPLIED;
+    const bool needs_noise =
+        supplied && (attack->kind == BRACE_ATTACK_GAUSSIAN || attack->kind == BRACE_ATTACK_SPARSE_NOISE);
+    const bool needs_unif = supplied && attack->kind == BRACE_ATTACK_SPARSE_NOISE;
     if (needs_noise && (!attack->noise || !d_noise_stage || attack->noise_ld < ctx->d)) return BRACE_ERR_INVALID_ARG;
     if (needs_unif && (!attack->uniform || !d_uniform_stage || attack->uniform_ld < ctx->d))
       return BRACE_ERR_INVALID_ARG;
@@ -897,6 +965,7 @@ int brace_aggregate_static(int32_t n, int64_t d, const brace_params* params, con
   if (2 * one_set > kStaticScratchBytes) return BRACE_ERR_WORKSPACE;
 
   brace_ctx ctx;                       // host stack only; its vectors stay empty
+  ctx.no_ctx_call = true;
   ctx.n = n;
   ctx.f = 0;
   ctx.d = d;
@@ -912,8 +981,13 @@ int brace_aggregate_static(int32_t n, int64_t d, const brace_params* params, con
   if (rc != BRACE_OK) return rc;
   if (!fused_layout_ok(&ctx, d_updates, ld, d_out, out_ld)) return BRACE_ERR_UNSUPPORTED;
   void* scratch = nullptr;
-  cudaError_t err = static_scratch_for_current_device(&scratch);
-  if (err != cudaSuccess) return BRACE_ERR_CUDA;
+  cudaError_t err = cudaGetSymbolAddress(&scratch, g_static_scratch);
+  if (err != cudaSuccess) return cuda_fail(&ctx, err);
+  if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255u) != 0) return cuda_fail(&ctx, cudaErrorInvalidSymbol);
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+    ctx.sm_count = sms;
   ctx.ws = static_cast<char*>(scratch);
   ctx.ws_bytes = kStaticScratchBytes;
   ctx.mail[0] = ctx.ws;

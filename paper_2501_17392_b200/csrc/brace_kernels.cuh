@@ -39,7 +39,8 @@ __device__ __forceinline__ int sgn1(float x, int zs) {
 // next hop's CTAs may start while the current hop drains.  pdl_wait() returns
 // once every kernel launched before this one on the stream has completed and
 // its writes are visible; before it a kernel may only read memory that no
-// earlier kernel of the round writes (the update matrix, from hop 1 on).
+// earlier kernel of the round writes (the update matrix, from hop 1 on: hop 0
+// waits for the matrix's producer before it lets hop 1 start).
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
@@ -89,8 +90,10 @@ rs_step_sign_kernel(Part pt, const float* __restrict__ U, int64_t ld, const P* _
   const float* ur = U + (int64_t)r * ld + b;
   const P* in = mail_in + (int64_t)c * seg_pad;
   P* out = mail_out + (int64_t)r * seg_pad;
+  // Hop 0 lets the next hop start only after it has itself seen the producer of the update
+  // matrix complete: hop 1 reads its updates before its own wait, and that wait covers hop 0 only.
+  if (step == 0) pdl_wait();
   pdl_launch_dependents();
-  if (step == 0) pdl_wait();                      // whoever produced the updates must have finished
   if (VPT > 0) {
     constexpr int V = VPT > 0 ? VPT : 1;
     const int64_t base = (int64_t)blockIdx.x * (256 * V) + threadIdx.x;
@@ -159,8 +162,8 @@ rs_step_sum_kernel(Part pt, const float* __restrict__ U, int64_t ld, const float
   const float* in = (step == 0) ? uc : mail_in + (int64_t)c * seg_pad;
   float* out = mail_out + (int64_t)r * seg_pad;
   const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (step == 0) pdl_wait();                        // see rs_step_sign_kernel
   pdl_launch_dependents();
-  if (step == 0) pdl_wait();
   if (VEC) {
     const int64_t i = t * 4;
     if (i + 4 <= L) {
@@ -387,12 +390,12 @@ struct FusedArgs {
   int owner_only;   // sign rules: write the consensus bits to the owner's row only (a share-only kernel follows)
 };
 
-template <typename P, int VPT, int UNR, bool ZS>
-__global__ void __launch_bounds__(256)
+template <typename P, int VPT, int UNR, bool ZS, int TPB>
+__global__ void __launch_bounds__(TPB)
 fused_sign_kernel(const FusedArgs a) {
   static_assert(VPT >= 1 && VPT <= 8, "tile width");
-  constexpr int TILE = 256 * 4 * VPT;
-  constexpr int WPT = 32 * VPT;                    // output words per tile
+  constexpr int TILE = TPB * 4 * VPT;
+  constexpr int WPT = (TPB / 8) * VPT;             // output words per tile
   __shared__ uint32_t sm_words[WPT];
   const Part pt = a.pt;
   const int n = pt.n;
@@ -413,7 +416,7 @@ fused_sign_kernel(const FusedArgs a) {
     int acc[VPT][4];
 #pragma unroll
     for (int v = 0; v < VPT; ++v) {
-      off[v] = t0 + (int64_t)(v * 256 + tid) * 4;
+      off[v] = t0 + (int64_t)(v * TPB + tid) * 4;
       const int64_t rem = L - off[v];
       nv[v] = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
       acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0;
@@ -472,7 +475,7 @@ fused_sign_kernel(const FusedArgs a) {
       word |= __shfl_xor_sync(0xffffffffu, word, 1);
       word |= __shfl_xor_sync(0xffffffffu, word, 2);
       word |= __shfl_xor_sync(0xffffffffu, word, 4);
-      if ((lane & 7) == 0) sm_words[v * 32 + warp * 4 + (lane >> 3)] = word;
+      if ((lane & 7) == 0) sm_words[v * (TPB / 8) + warp * 4 + (lane >> 3)] = word;
     }
     __syncthreads();
     const int64_t left = L - t0;
@@ -484,7 +487,7 @@ fused_sign_kernel(const FusedArgs a) {
       if (a.owner_only) {                            // client j-1 owns sub-vector j (Phase III is local to the owner)
         if (tid < WPT) out[(int64_t)(j == 0 ? n - 1 : j - 1) * a.out_ld + wb + w] = val;
       } else {
-        for (int row = tid / WPT; row < n; row += 256 / WPT) out[(int64_t)row * a.out_ld + wb + w] = val;
+        for (int row = tid / WPT; row < n; row += TPB / WPT) out[(int64_t)row * a.out_ld + wb + w] = val;
       }
     }
     __syncthreads();
@@ -721,6 +724,116 @@ inject_stats_kernel(int kind, const int* __restrict__ ids, int f, int n, const f
 }
 
 
+// ---------------------------------------------------------------------------
+// Random draws made inside the library.  The generator is counter-based, so a
+// draw is a pure function of (seed, round, client, coordinate, stream) and no
+// state travels between launches: Philox4x32 with 10 rounds (Salmon et al.,
+// "Parallel random numbers: as easy as 1, 2, 3", SC'11), written here from its
+// definition.  Four coordinates share one call: block q = k / 4 uses key
+// (seed lo, seed hi) and counter (q lo, q hi, client, round * 256 + stream);
+// word k % 4 belongs to coordinate k.
+// ---------------------------------------------------------------------------
+constexpr uint32_t kStreamUniform = 0;    // top 24 bits of the word, times 2^-24: uniform in [0, 1)
+constexpr uint32_t kStreamNormal = 1;     // words (a, b) of a coordinate pair -> two normals (Box-Muller)
+
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 key) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    c = make_uint4(hi1 ^ c.y ^ key.x, lo1, hi0 ^ c.w ^ key.y, lo0);
+    key.x += 0x9E3779B9u;
+    key.y += 0xBB67AE85u;
+  }
+  return c;
+}
+
+__device__ __forceinline__ uint4 draw_block(uint64_t seed, uint32_t round, uint32_t client, uint32_t stream, int64_t q) {
+  return philox4x32_10(make_uint4((uint32_t)q, (uint32_t)((uint64_t)q >> 32), client, round * 256u + stream),
+                       make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)));
+}
+
+__device__ __forceinline__ float uniform_from_word(uint32_t w) { return __fmul_rn((float)(w >> 8), 5.9604644775390625e-8f); }
+
+// Box-Muller in float32: u1 = ((a >> 8) + 1) / 2^24 in (0, 1], u2 = (b >> 8) / 2^24;
+// radius = sqrt(-2 ln u1); (radius cos 2 pi u2, radius sin 2 pi u2).
+__device__ __forceinline__ void normal_pair(uint32_t a, uint32_t b, float& z0, float& z1) {
+  const float u1 = __fmul_rn((float)((a >> 8) + 1u), 5.9604644775390625e-8f);
+  const float two_u2 = __fmul_rn((float)(b >> 8), 1.1920928955078125e-7f);   // exact
+  const float radius = __fsqrt_rn(__fmul_rn(-2.0f, logf(u1)));
+  float s, c;
+  sincospif(two_u2, &s, &c);
+  z0 = __fmul_rn(radius, c);
+  z1 = __fmul_rn(radius, s);
+}
+
+// Rows of raw draws, for inspection and as a building block of synthetic inputs:
+// out[i][k] = mu + sigma * z (what = 1, standard normal z) or the uniform itself
+// (what = 0).  Row i belongs to client first_client + i.  grid = (blocks of 4
+// coordinates, rows).
+__global__ void __launch_bounds__(256)
+draw_matrix_kernel(int what, uint64_t seed, uint32_t round, int first_client, float* __restrict__ out, int64_t ld,
+                   int64_t d, float mu, float sigma, int vec) {
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t k = q * 4;
+  if (k >= d) return;
+  const uint32_t client = (uint32_t)(first_client + (int)blockIdx.y);
+  float v[4];
+  if (what == 0) {
+    const uint4 w = draw_block(seed, round, client, kStreamUniform, q);
+    v[0] = uniform_from_word(w.x); v[1] = uniform_from_word(w.y);
+    v[2] = uniform_from_word(w.z); v[3] = uniform_from_word(w.w);
+  } else {
+    const uint4 w = draw_block(seed, round, client, kStreamNormal, q);
+    normal_pair(w.x, w.y, v[0], v[1]);
+    normal_pair(w.z, w.w, v[2], v[3]);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = __fadd_rn(mu, __fmul_rn(sigma, v[e]));
+  }
+  float* dst = out + (int64_t)blockIdx.y * ld + k;
+  if (vec && k + 4 <= d) {
+    *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+  } else {
+    for (int e = 0; e < 4 && k + e < d; ++e) dst[e] = v[e];
+  }
+}
+
+// Alterations that consume randomness, drawing it here instead of reading
+// pre-drawn matrices: kind 2 (b = sigma * z) and kind 5 (b = sigma * z where the
+// coordinate's uniform is below prob, else 0).  Only the 4*f*d bytes of the
+// Byzantine rows move.  For kind 5 the normals of a block are computed only if
+// one of its four coordinates passes the test.  grid = (blocks of 4
+// coordinates, f Byzantine rows).
+__global__ void __launch_bounds__(256)
+inject_generated_kernel(int kind, const int* __restrict__ ids, float* __restrict__ Uo, int64_t ld_u, int64_t d,
+                        uint64_t seed, uint32_t round, float sigma, float prob, int vec) {
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t k = q * 4;
+  if (k >= d) return;
+  const int id = ids[blockIdx.y];
+  float v[4] = {0.f, 0.f, 0.f, 0.f};
+  bool take[4] = {true, true, true, true};
+  if (kind != 2) {
+    const uint4 w = draw_block(seed, round, (uint32_t)id, kStreamUniform, q);
+    take[0] = uniform_from_word(w.x) < prob; take[1] = uniform_from_word(w.y) < prob;
+    take[2] = uniform_from_word(w.z) < prob; take[3] = uniform_from_word(w.w) < prob;
+  }
+  if (take[0] | take[1] | take[2] | take[3]) {
+    const uint4 w = draw_block(seed, round, (uint32_t)id, kStreamNormal, q);
+    float z[4];
+    if (take[0] | take[1]) normal_pair(w.x, w.y, z[0], z[1]);
+    if (take[2] | take[3]) normal_pair(w.z, w.w, z[2], z[3]);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = take[e] ? __fmul_rn(sigma, z[e]) : 0.0f;
+  }
+  float* dst = Uo + (int64_t)id * ld_u + k;
+  if (vec && k + 4 <= d) {
+    __stcs(reinterpret_cast<float4*>(dst), make_float4(v[0], v[1], v[2], v[3]));
+  } else {
+    for (int e = 0; e < 4 && k + e < d; ++e) dst[e] = v[e];
+  }
+}
+
 // 128-bit variant of the element-wise alterations (rows 16-byte aligned).
 __global__ void __launch_bounds__(256)
 inject_elementwise_vec_kernel(int kind, const int* __restrict__ ids, const float* H, int64_t ld_h, float* Uo,
@@ -883,32 +996,53 @@ __global__ void inject_stats_smem_kernel(int kind, const int* __restrict__ ids, 
   }
 }
 
-// Register-resident variant of the statistics kernel for up to 128 honest rows:
+// Register-resident variant of the statistics kernel for up to 127 honest rows:
 // a thread owns one coordinate, requests all of its honest values at once (they
 // stay in registers), then runs the float64 sum and the float64 deviations over
-// them -- the second pass costs no memory traffic at all.  MFULL rows (a
-// multiple of 8) are handled without predicates, up to 7 more with.  Row byte
-// offsets travel as a kernel parameter so that, with the loops unrolled, every
-// row address is one 64-bit add with a constant operand.
+// them -- the second pass costs no memory traffic at all.  MFULL rows are
+// handled without predicates, up to MTAIL more with.
+//
+// The kernel is bound by instruction issue at low occupancy (the values of a
+// coordinate fill most of a thread's registers), so what counts is instructions
+// per element.  Two ways to address the rows:
+//   STRIDED  honest rows are consecutive clients: row r is at base + r * stride,
+//            one 32x32+64-bit multiply-add with r a constant; the Byzantine rows
+//            are consecutive too and are stored by stepping a pointer;
+//   table    row byte offsets travel as a kernel parameter (constant bank), the
+//            Byzantine ids are read from the workspace.
 struct HonestRows {
   int64_t byte_off[128];
 };
 
-template <int MFULL>
-__global__ void __launch_bounds__(128, (MFULL <= 24 ? 8 : (MFULL <= 40 ? 6 : (MFULL <= 56 ? 5 : (MFULL <= 80 ? 4 : (MFULL <= 96 ? 3 : 2))))))
-inject_stats_reg_kernel(int kind, const __grid_constant__ HonestRows rows, const int* __restrict__ ids, int f, int m,
-                        const float* H, float* Uo, int64_t ld_u, int64_t d, float scale, float kappa) {
-  constexpr int MTAIL = 7;
+#ifndef BRACE_STATS_MINB_80
+#define BRACE_STATS_MINB_80 4
+#endif
+
+constexpr int stats_min_blocks(int mfull) {
+  return mfull <= 24 ? 8 : (mfull <= 40 ? 6 : (mfull <= 56 ? 5 : (mfull <= 80 ? BRACE_STATS_MINB_80 : (mfull <= 96 ? 3 : 2))));
+}
+
+template <int MFULL, int MTAIL, bool STRIDED>
+__global__ void __launch_bounds__(128, stats_min_blocks(MFULL))
+inject_stats_reg_kernel(int kind, const __grid_constant__ HonestRows rows, uint32_t stride_bytes,
+                        const int* __restrict__ ids, int f, int m, const float* H, float* Uo, int64_t ld_u, int64_t d,
+                        float scale, float kappa) {
   const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (k >= d) return;
+  // STRIDED: H points at the first honest row, Uo at the first Byzantine row
   const char* src = reinterpret_cast<const char*>(H + k);
-  const int tail = m - MFULL;                        // 0..7 rows beyond the unpredicated ones
+  const int tail = m - MFULL;                        // 0..MTAIL rows beyond the unpredicated ones
+  auto row_ptr = [&](int r) -> const float* {
+    return reinterpret_cast<const float*>(STRIDED ? src + (uint64_t)stride_bytes * (uint32_t)r : src + rows.byte_off[r]);
+  };
   float x[MFULL + MTAIL];
 #pragma unroll
-  for (int r = 0; r < MFULL; ++r) x[r] = __ldcs(reinterpret_cast<const float*>(src + rows.byte_off[r]));
+  for (int r = 0; r < MFULL; ++r) x[r] = __ldcs(row_ptr(r));
 #pragma unroll
-  for (int r = 0; r < MTAIL; ++r)
-    x[MFULL + r] = (r < tail) ? __ldcs(reinterpret_cast<const float*>(src + rows.byte_off[MFULL + r])) : 0.0f;
+  for (int r = 0; r < MTAIL; ++r) {
+    x[MFULL + r] = 0.0f;
+    if (r < tail) x[MFULL + r] = __ldcs(row_ptr(MFULL + r));
+  }
   double tot = 0.0;
 #pragma unroll
   for (int r = 0; r < MFULL; ++r) tot = __dadd_rn(tot, (double)x[r]);
@@ -923,17 +1057,28 @@ inject_stats_reg_kernel(int kind, const __grid_constant__ HonestRows rows, const
   } else {
     double sq = 0.0;
 #pragma unroll
-    for (int r = 0; r < MFULL + MTAIL; ++r) {
-      if (r < MFULL || r - MFULL < tail) {
-        asm volatile("" : "+f"(x[r]));               // convert again rather than keep 2 registers per value
-        const double dev = __dsub_rn((double)x[r], mean);
+    for (int r = 0; r < MFULL; ++r) {
+      asm volatile("" : "+f"(x[r]));                 // convert again rather than keep 2 registers per value
+      const double dev = __dsub_rn((double)x[r], mean);
+      sq = __dadd_rn(sq, __dmul_rn(dev, dev));
+    }
+#pragma unroll
+    for (int r = 0; r < MTAIL; ++r) {
+      if (r < tail) {
+        asm volatile("" : "+f"(x[MFULL + r]));
+        const double dev = __dsub_rn((double)x[MFULL + r], mean);
         sq = __dadd_rn(sq, __dmul_rn(dev, dev));
       }
     }
     vec = __dsub_rn(mean, __dmul_rn((double)kappa, __dsqrt_rn(__ddiv_rn(sq, dm))));
   }
   const float v = __double2float_rn(vec);
-  for (int bq = 0; bq < f; ++bq) Uo[(int64_t)ids[bq] * ld_u + k] = v;
+  if (STRIDED) {
+    float* dst = Uo + k;
+    for (int bq = 0; bq < f; ++bq, dst += ld_u) *dst = v;
+  } else {
+    for (int bq = 0; bq < f; ++bq) Uo[(int64_t)ids[bq] * ld_u + k] = v;
+  }
 }
 
 // ---------------------------------------------------------------------------

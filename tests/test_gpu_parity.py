@@ -573,6 +573,33 @@ def test_attack_injection_and_pipeline(name, d, ids):
     ctx.close()
 
 
+@pytest.mark.parametrize("n,f", [(100, 20), (9, 2), (37, 5), (128, 1), (12, 11)])
+def test_mean_shift_statistics_special_values(n, f):
+    """Honest rows sprinkled with +-0, denormals, +-FLT_MAX, +-Inf and NaN: the statistics kernel widens
+    float32 to float64 with integer operations where every input of a coordinate is a normal number and
+    falls back to the conversion instruction elsewhere; both routes must give the oracle's bits (a
+    coordinate whose oracle value is NaN must be NaN)."""
+    d, ld = 6_000, 6_016
+    H = W.edge_value_updates(n, d, seed=n, ld=ld)
+    Hn = H.numpy()
+    Hn[:, : d // 2] = np.where(np.isfinite(Hn[:, : d // 2]), Hn[:, : d // 2], np.float32(0.25))   # first half: no Inf / NaN
+    Hn[:, : d // 4] = np.where(np.abs(Hn[:, : d // 4]) > 1e30, np.float32(-3.0), Hn[:, : d // 4])  # first quarter: no overflow
+    g = torch.Generator().manual_seed(7 * n)
+    Hn[:, 100:1100] = torch.empty((n, 1000)).normal_(0.0, 0.01, generator=g).numpy()               # all-normal columns
+    for kind, kw in ((B.ATTACK_MEAN_SHIFT, dict(kappa=3.0)), (B.ATTACK_SCALED_MEAN, dict(scale=-5.0))):
+        ctx = B.Brace(n, f, d)
+        U = H.cuda()
+        ctx.inject_attack(B.make_attack(kind, **kw), U, U)
+        with np.errstate(all="ignore"):
+            exp = O.inject_attack(kind, Hn[:, :d], list(range(f)), **kw)
+        got = U.cpu().numpy()[:, :d]
+        nan = np.isnan(exp)
+        assert np.array_equal(np.isnan(got), nan)
+        assert nan[:, : d // 2].sum() == 0 and nan.sum() > 0
+        assert np.array_equal(got.view(np.uint32)[~nan], exp.view(np.uint32)[~nan])
+        ctx.close()
+
+
 @pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
 def test_attack_injection_unaligned_rows(name):
     """Row strides that are not multiples of 4 take the scalar kernels; same bits."""

@@ -478,3 +478,131 @@ def test_coordinate_median_and_trimmed_mean_against_library_routines():
     assert O.coordinate_median(V).tolist() == O.coordinate_median(U).tolist()
     with pytest.raises(ValueError):
         O.coordinate_trimmed_mean(U, 2)
+
+
+# ---------------------------------------------------------------- random draws of the attacks
+def _kat_rows():
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt")
+    rows, numer = [], None
+    with open(path) as fh:
+        for line in fh:
+            line = line.strip()
+            if line.startswith("# uniform_numerators:"):
+                numer = [int(v) for v in line.split(":")[1].split()]
+            if not line or line.startswith("#"):
+                continue
+            rows.append([int(v, 16) for v in line.split()])
+    return rows, numer
+
+
+def test_philox_known_answer_vectors():
+    """The published known-answer vectors of Philox4x32-10."""
+    rows, _ = _kat_rows()
+    assert len(rows) == 3
+    for r in rows:
+        got = O.philox4x32_10([np.array([c], dtype=np.uint32) for c in r[0:4]], r[4:6])
+        assert [int(g[0]) for g in got] == r[6:10]
+    # vectorised over counters: same answers in one call
+    ctr = [np.array([r[i] for r in rows], dtype=np.uint32) for i in range(4)]
+    key = [np.array([r[4 + i] for r in rows], dtype=np.uint32) for i in range(2)]
+    got = O.philox4x32_10(ctr, key)
+    for t, r in enumerate(rows):
+        assert [int(g[t]) for g in got] == r[6:10]
+
+
+def test_draw_layout_counter_and_key_fields():
+    """Where seed, round, client, stream and coordinate go: block q = k div 4 -> counter
+    (q lo, q hi, client, round * 256 + stream), key (seed lo, seed hi); word k mod 4.
+    Philox itself is pinned by the known-answer vectors, so the field layout is checked
+    through it; the all-zero case is the first published vector."""
+    rows, numer = _kat_rows()
+    assert O.draw_words(0, 0, 0, O.STREAM_UNIFORM, 4).tolist() == rows[0][6:10]
+    u = O.draw_uniform(0, 0, 0, 4)
+    assert [int(round(float(x) * 2 ** 24)) for x in u] == numer
+    seed, rnd, client, stream, d = 0x299F31D0A4093822, 0x037073, 0x13198A2E, 0x44, 27
+    w = O.draw_words(seed, rnd, client, stream, d)
+    assert w.dtype == np.uint32 and w.shape == (d,)
+    for k in (0, 1, 5, 11, 24, 26):
+        q = k // 4
+        ref = O.philox4x32_10([np.array([v], dtype=np.uint32) for v in (q, 0, client, rnd * 256 + stream)],
+                              [seed & 0xFFFFFFFF, seed >> 32])
+        assert int(w[k]) == int(ref[k % 4][0])
+    # the third published vector has exactly this key, client word and round/stream word
+    assert rnd * 256 + stream == rows[2][3] and client == rows[2][2]
+    assert [seed & 0xFFFFFFFF, seed >> 32] == rows[2][4:6]
+    # every field matters, and a prefix does not depend on d
+    base = O.draw_words(5, 1, 2, 0, 64)
+    for other in (O.draw_words(6, 1, 2, 0, 64), O.draw_words(5 + (1 << 32), 1, 2, 0, 64), O.draw_words(5, 2, 2, 0, 64),
+                  O.draw_words(5, 1, 3, 0, 64), O.draw_words(5, 1, 2, 1, 64)):
+        assert (other != base).mean() > 0.9
+    assert np.array_equal(O.draw_words(5, 1, 2, 0, 13), base[:13])
+    assert np.array_equal(O.draw_words(5, 1, 2, 0, 21, start=40), base[40:61])         # a window of the same row
+    assert np.array_equal(O.draw_normal(5, 1, 2, 9, start=8), O.draw_normal(5, 1, 2, 17)[8:])
+    assert np.array_equal(O.draw_uniform(5, 1, 2, 9, start=8), O.draw_uniform(5, 1, 2, 17)[8:])
+    big = (1 << 34) + 8                                                                # block index needs its high word
+    hi = O.draw_words(5, 1, 2, 0, 4, start=big)
+    ref = O.philox4x32_10([np.array([v], dtype=np.uint32) for v in ((big // 4) & 0xFFFFFFFF, (big // 4) >> 32, 2, 256)], [5, 0])
+    assert [int(x) for x in hi] == [int(r[0]) for r in ref]
+    for bad in ((-1, 0, 0, 0), (1 << 64, 0, 0, 0), (0, 1 << 24, 0, 0), (0, 0, 0, 256)):
+        with pytest.raises(ValueError):
+            O.draw_words(bad[0], bad[1], bad[2], bad[3], 4)
+
+
+def test_uniform_and_normal_draws_have_their_distributions():
+    """Uniforms are multiples of 2^-24 in [0, 1); normals pass a Kolmogorov-Smirnov test against
+    scipy's normal distribution; different clients / rounds are uncorrelated."""
+    from scipy import stats
+    d = 400_001
+    u = O.draw_uniform(2501017392, 3, 7, d)
+    assert u.dtype == np.float32 and u.min() >= 0.0 and u.max() < 1.0
+    assert np.array_equal(u.astype(np.float64) * 2 ** 24, np.rint(u.astype(np.float64) * 2 ** 24))
+    assert stats.kstest(u.astype(np.float64), "uniform").pvalue > 1e-3
+    z = O.draw_normal(2501017392, 3, 7, d)
+    assert z.dtype == np.float32 and np.isfinite(z).all()
+    assert stats.kstest(z.astype(np.float64), "norm").pvalue > 1e-3
+    assert abs(float(z.mean())) < 0.01 and abs(float(z.var()) - 1.0) < 0.01
+    assert abs(np.corrcoef(z[0::2][: d // 2], z[1::2][: d // 2])[0, 1]) < 0.01       # the two outputs of a pair
+    z2 = O.draw_normal(2501017392, 3, 8, d)
+    z3 = O.draw_normal(2501017392, 4, 7, d)
+    assert abs(np.corrcoef(z, z2)[0, 1]) < 0.01 and abs(np.corrcoef(z, z3)[0, 1]) < 0.01
+    assert abs(np.corrcoef(z, u)[0, 1]) < 0.01
+
+
+def test_normal_draws_invert_to_their_words():
+    """Box-Muller run backwards: from a pair (z0, z1), exp(-(z0^2 + z1^2) / 2) is u1 and the angle
+    atan2(z1, z0) / (2 pi) is u2 -- both must be the 24-bit fractions of the pair's two words.
+    A swapped cos / sin, a wrong radius or the wrong words fail this."""
+    seed, rnd, client, d = 99, 5, 11, 20_000
+    z = O.draw_normal(seed, rnd, client, d).astype(np.float64).reshape(-1, 2)
+    w = O.draw_words(seed, rnd, client, O.STREAM_NORMAL, d).reshape(-1, 2)
+    u1 = ((w[:, 0] >> 8).astype(np.float64) + 1.0) / 2 ** 24
+    u2 = (w[:, 1] >> 8).astype(np.float64) / 2 ** 24
+    r2 = (z * z).sum(1)
+    assert np.allclose(np.exp(-0.5 * r2), u1, rtol=2e-6, atol=0)
+    ang = np.mod(np.arctan2(z[:, 1], z[:, 0]) / (2 * np.pi), 1.0)
+    err = np.abs(ang - u2)
+    err = np.minimum(err, 1.0 - err)
+    ok = r2 > 1e-6                                     # a zero radius has no angle
+    assert err[ok].max() < 1e-6
+    # odd d: the last coordinate is the first output of its pair
+    assert np.array_equal(O.draw_normal(seed, rnd, client, 7), O.draw_normal(seed, rnd, client, 8)[:7])
+
+
+def test_cospi_sinpi_exact_at_quarter_turns():
+    x = np.array([0.0, 0.25, 0.5, 0.75, 1.0, 1.25, 1.5, 1.75, 1.0 / 3.0])
+    c, s = O._cospi_sinpi(x)
+    h = math.sqrt(0.5)
+    assert np.allclose(c[:8], [1, h, 0, -h, -1, -h, 0, h], rtol=1e-15, atol=0)
+    assert np.allclose(s[:8], [0, h, 1, h, 0, -h, -1, -h], rtol=1e-15, atol=0)
+    assert c[2] == 0.0 and c[6] == 0.0 and s[0] == 0.0 and s[4] == 0.0       # exact zeros, not 6e-17
+    assert abs(c[8] - 0.5) < 1e-15
+
+
+def test_attack_draws_shapes_and_rows():
+    noise, unif = O.attack_draws(O.ATTACK_SPARSE_NOISE, 7, 2, [5, 1], 33)
+    assert noise.shape == (2, 33) and unif.shape == (2, 33)
+    assert np.array_equal(noise[1], O.draw_normal(7, 2, 1, 33)) and np.array_equal(unif[0], O.draw_uniform(7, 2, 5, 33))
+    noise, unif = O.attack_draws(O.ATTACK_GAUSSIAN, 7, 2, [0], 8)
+    assert unif is None and noise.shape == (1, 8)
+    assert O.attack_draws(O.ATTACK_MEAN_SHIFT, 7, 2, [0], 8) == (None, None)
