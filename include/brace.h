@@ -313,15 +313,21 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
                         int64_t* len, int32_t* segment, int32_t* entry_bytes);
 
 /* Expert knob for measurements: pick the fused kernel's shape.  fused_variant
- * 0 = library default, 1..5 = (float4 per thread per client, clients
- * prefetched) in {(1,8),(2,4),(1,4),(2,8),(1,16)}; fused_grid = 0 launches one
- * CTA per tile, > 0 caps the grid (CTAs then loop over tiles).  Adding 10, 20
- * or 40 to fused_variant makes the share-reduce hop kernel process 1, 2 or 4
- * float4 per thread (default: 4, fewer for short sub-vectors).  On large
- * problems (n*d >= 2^27) the fused kernel writes each sub-vector's bits to its
- * owner's row and one share-only launch spreads them to the other rows; adding
- * 1000 forces that at any size, adding 2000 makes the fused kernel write all n
- * rows itself.  Results do not depend on any of these. */
+ * 0 = library default; 1..5 and 7 = (float4 per thread per client, clients
+ * prefetched, threads per CTA) in {(1,8,256),(2,4,256),(1,4,256),(2,8,256),
+ * (1,16,256)} and (1,8,128); 6, 8, 9 = the software-pipelined kernel with
+ * persistent CTAs and (clients per batch, threads per CTA) in {(4,128),(8,128),
+ * (8,256)}.  fused_grid = 0 launches one CTA per tile (pipelined kernel: as many
+ * CTAs as stay resident), > 0 caps the grid (CTAs then loop over tiles).
+ * Adding 10, 20 or 40 to fused_variant makes the share-reduce hop kernel process
+ * 1, 2 or 4 float4 per thread (default: 4, fewer for short sub-vectors); adding
+ * 100, 200 or 400 picks the staged statistics kernel with 1, 2 or 4 floats per
+ * thread, 800 makes the register-resident statistics kernel address rows through
+ * its offset table even when they are consecutive.  On large problems
+ * (n*d >= 2^27) the fused kernel writes each sub-vector's bits to its owner's row
+ * and one share-only launch spreads them to the other rows; adding 1000 forces
+ * that at any size, adding 2000 makes the fused kernel write all n rows itself.
+ * Results do not depend on any of these. */
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid);
 
 /* Bytes of mailbox scratch built into the library for brace_aggregate_static. */

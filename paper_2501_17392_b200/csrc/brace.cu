@@ -327,6 +327,21 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
       else    fused_sign_kernel<int16_t, VPT, UNR, false, TPB><<<g, TPB, 0, st>>>(a);           \
     }                                                                                           \
   } while (0)
+#define BRACE_FUSED_PIPE(UNR, TPB, CTAS)                                                        \
+  do {                                                                                          \
+    fused_geometry(ctx, a, (int64_t)TPB * 4);                                                   \
+    int64_t gp = (int64_t)ctx->sm_count * CTAS;      /* persistent: what fits on the device */  \
+    if (ctx->fused_grid > 0) gp = ctx->fused_grid;                                              \
+    if (gp > a.units) gp = a.units;                                                             \
+    const unsigned g = (unsigned)(gp > 0 ? gp : 1);                                             \
+    if (ctx->entry_bytes == 1) {                                                                \
+      if (zs) fused_sign_pipe_kernel<int8_t, UNR, true, TPB><<<g, TPB, 0, st>>>(a);             \
+      else    fused_sign_pipe_kernel<int8_t, UNR, false, TPB><<<g, TPB, 0, st>>>(a);            \
+    } else {                                                                                    \
+      if (zs) fused_sign_pipe_kernel<int16_t, UNR, true, TPB><<<g, TPB, 0, st>>>(a);            \
+      else    fused_sign_pipe_kernel<int16_t, UNR, false, TPB><<<g, TPB, 0, st>>>(a);           \
+    }                                                                                           \
+  } while (0)
 #define BRACE_FUSED_SUM(VPT, UNR)                                                               \
   do {                                                                                          \
     fused_geometry(ctx, a, (int64_t)256 * 4 * VPT);                                             \
@@ -345,14 +360,15 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
       case 3: BRACE_FUSED_SIGN(1, 4, 256); break;
       case 4: BRACE_FUSED_SIGN(2, 8, 256); break;
       case 5: BRACE_FUSED_SIGN(1, 16, 256); break;
-      case 6: BRACE_FUSED_SIGN(1, 24, 256); break;
+      case 6: BRACE_FUSED_PIPE(4, 128, 5); break;
       case 7: BRACE_FUSED_SIGN(1, 8, 128); break;
-      case 8: BRACE_FUSED_SIGN(1, 16, 128); break;
-      case 9: BRACE_FUSED_SIGN(1, 24, 128); break;
+      case 8: BRACE_FUSED_PIPE(8, 128, 4); break;
+      case 9: BRACE_FUSED_PIPE(8, 256, 2); break;
       default: BRACE_FUSED_SIGN(1, 8, 256); break;
     }
   }
 #undef BRACE_FUSED_SIGN
+#undef BRACE_FUSED_PIPE
 #undef BRACE_FUSED_SUM
   int rc = check_launch(ctx);
   if (rc != BRACE_OK || !spread) return rc;
@@ -465,14 +481,14 @@ int inject_impl(brace_ctx* ctx, const brace_attack* atk, const float* H, int64_t
       bool strided = (ld_h * 4 < ((int64_t)1 << 32)) && ctx->stats_table == 0;
       for (int r = 1; r < m && strided; ++r) strided = ids[(size_t)f + r] == ids[(size_t)f] + r;
       for (int b = 1; b < f && strided; ++b) strided = ids[(size_t)b] == ids[0] + b;
-      const unsigned blocks = tiles(ctx->d, 128);
+      const unsigned blocks = tiles(ctx->d, kStatsThreads);
       if (strided) {
         const float* H0 = H + (int64_t)ids[(size_t)f] * ld_h;
         float* U0 = Uo + (int64_t)ids[0] * ld_u;
         HonestRows none{};
 #define BRACE_STATS_REG(MFULL)                                                                               \
   case MFULL:                                                                                                \
-    inject_stats_reg_kernel<MFULL, 3, true><<<blocks, 128, 0, st>>>(kind, none, (uint32_t)(ld_h * 4), nullptr, f, m, \
+    inject_stats_reg_kernel<MFULL, 3, true><<<blocks, kStatsThreads, 0, st>>>(kind, none, (uint32_t)(ld_h * 4), nullptr, f, m, \
                                                                     H0, U0, ld_u, ctx->d, atk->scale, atk->kappa);    \
     break
         switch (m / 4 * 4) {
@@ -493,7 +509,7 @@ int inject_impl(brace_ctx* ctx, const brace_attack* atk, const float* H, int64_t
         rows.byte_off[r] = (int64_t)ids[(size_t)f + (size_t)(r < m ? r : m - 1)] * ld_h * 4;
 #define BRACE_STATS_REG(MFULL)                                                                                \
   case MFULL:                                                                                                 \
-    inject_stats_reg_kernel<MFULL, 7, false><<<blocks, 128, 0, st>>>(kind, rows, 0u, ctx->d_ids, f, m, H, Uo, ld_u, \
+    inject_stats_reg_kernel<MFULL, 7, false><<<blocks, kStatsThreads, 0, st>>>(kind, rows, 0u, ctx->d_ids, f, m, H, Uo, ld_u, \
                                                                      ctx->d, atk->scale, atk->kappa);         \
     break
       switch (m / 8 * 8) {
@@ -814,14 +830,14 @@ int brace_coordinate_stat(brace_ctx* ctx, int32_t kind, int32_t trim, const floa
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const unsigned blocks = tiles(ctx->d, 128);
   const int n = ctx->n;
-#define BRACE_STAT(NP) \
-  coordinate_stat_kernel<NP><<<blocks, 128, 0, st>>>(kind, trim, n, d_updates, ld, d_result, ctx->d)
-  if (n <= 4) BRACE_STAT(4);
-  else if (n <= 8) BRACE_STAT(8);
-  else if (n <= 16) BRACE_STAT(16);
-  else if (n <= 32) BRACE_STAT(32);
-  else if (n <= 64) BRACE_STAT(64);
-  else BRACE_STAT(128);
+#define BRACE_STAT(NB) \
+  case NB: coordinate_stat_kernel<NB><<<blocks, 128, 0, st>>>(kind, trim, n, d_updates, ld, d_result, ctx->d); break
+  switch (n <= 4 ? 4 : (n + 7) / 8 * 8) {            // n rounded up to a multiple of 8 (4 for the smallest)
+    BRACE_STAT(4); BRACE_STAT(8); BRACE_STAT(16); BRACE_STAT(24); BRACE_STAT(32); BRACE_STAT(40); BRACE_STAT(48);
+    BRACE_STAT(56); BRACE_STAT(64); BRACE_STAT(72); BRACE_STAT(80); BRACE_STAT(88); BRACE_STAT(96); BRACE_STAT(104);
+    BRACE_STAT(112); BRACE_STAT(120);
+    default: BRACE_STAT(128);
+  }
 #undef BRACE_STAT
   return check_launch(ctx);
 }

@@ -494,6 +494,161 @@ fused_sign_kernel(const FusedArgs a) {
   }
 }
 
+// Software-pipelined form of the fused round for problems of a few L2 sizes or
+// less, where a launch is too short for the CTAs' load and compute phases to
+// drift apart on their own.  A persistent CTA walks its tiles (tile u, then
+// u + gridDim.x, ...) as one flat sequence of client batches; the loads of the
+// next batch -- of the same tile or of the CTA's next tile -- are issued before
+// the current batch is consumed, so every warp always has UNR loads in flight.
+// Tile width is TPB * 4 coordinates (one float4 per thread per client).  The
+// result and the two surviving mailbox states are those of fused_sign_kernel.
+template <typename P, int UNR, bool ZS, int TPB>
+__global__ void __launch_bounds__(TPB)
+fused_sign_pipe_kernel(const FusedArgs a) {
+  constexpr int TILE = TPB * 4;
+  constexpr int WPT = TPB / 8;                       // output words per tile
+  __shared__ uint32_t sm_words[WPT];
+  const Part pt = a.pt;
+  const int n = pt.n;
+  const int nb = (n + UNR - 1) / UNR;                // client batches per tile
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* __restrict__ U = a.U;
+  uint32_t* __restrict__ out = reinterpret_cast<uint32_t*>(a.out);
+  const uint32_t tps = (uint32_t)a.tiles_per_seg;
+  const bool small = a.units < ((int64_t)1 << 31) && (int64_t)n * pt.Q < ((int64_t)1 << 31);
+
+  struct Tile {
+    int64_t b;      // first coordinate of the sub-vector
+    int64_t off;    // this thread's first coordinate within the sub-vector
+    int j;          // sub-vector
+    int nv;         // valid coordinates of this thread's float4 (0..4)
+    int left;       // coordinates of the sub-vector from the tile's start on (capped at TILE)
+  };
+  // first non-empty tile at or after u in this CTA's sequence; false when the sequence is exhausted
+  auto find = [&](int64_t& u, Tile& t) -> bool {
+    for (; u < a.units; u += gridDim.x) {
+      int j, k;
+      int64_t b, e;
+      if (small) {                                   // 32-bit divisions
+        j = (int)((uint32_t)u / tps);
+        k = (int)((uint32_t)u - (uint32_t)j * tps);
+        const uint32_t q = (uint32_t)pt.Q, un = (uint32_t)n;
+        b = pt.G * (int64_t)(((uint32_t)j * q) / un);
+        e = pt.G * (int64_t)(((uint32_t)(j + 1) * q) / un);
+        b = b < pt.d ? b : pt.d;
+        e = (j + 1 == n || e > pt.d) ? pt.d : e;
+      } else {
+        j = (int)(u / tps);
+        k = (int)(u % tps);
+        b = pt.begin(j);
+        e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+      }
+      const int64_t L = e - b, t0 = (int64_t)k * TILE;
+      if (t0 >= L) continue;
+      t.b = b;
+      t.j = j;
+      t.off = t0 + (int64_t)tid * 4;
+      const int64_t rem = L - t.off;
+      t.nv = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
+      t.left = (int)(L - t0 < TILE ? L - t0 : TILE);
+      return true;
+    }
+    return false;
+  };
+
+  // ---- loader state
+  int64_t ul = blockIdx.x;
+  Tile tl;
+  bool have_l = find(ul, tl);
+  int bl = 0, cl = have_l ? tl.j : 0;                // batch within the tile, client of the next load
+  // ---- consumer state
+  int64_t uc = ul;
+  Tile tc = tl;
+  bool have_c = have_l;
+  int bc = 0, cc = cl;
+  int acc[4] = {0, 0, 0, 0};
+
+  auto issue = [&](float4 (&x)[UNR]) {
+    if (!have_l) return;
+    const float* p = U + tl.b + tl.off;
+#pragma unroll
+    for (int q = 0; q < UNR; ++q) {
+      if (bl * UNR + q < n) {
+        x[q] = tl.nv > 0 ? ld_stream(p + (int64_t)cl * a.ld) : make_float4(0.f, 0.f, 0.f, 0.f);
+        cl = next_client(cl, n);
+      }
+    }
+    if (++bl == nb) {
+      bl = 0;
+      ul += gridDim.x;
+      have_l = find(ul, tl);
+      cl = have_l ? tl.j : 0;
+    }
+  };
+
+  auto consume = [&](float4 (&x)[UNR]) {
+#pragma unroll
+    for (int q = 0; q < UNR; ++q) {
+      const int i = bc * UNR + q;
+      if (i < n) {
+        acc[0] += sgn1<ZS>(x[q].x, a.zs);
+        acc[1] += sgn1<ZS>(x[q].y, a.zs);
+        acc[2] += sgn1<ZS>(x[q].z, a.zs);
+        acc[3] += sgn1<ZS>(x[q].w, a.zs);
+        if (i >= 1 && i >= n - 2) {                  // hop s = i-1 lands in client cc's mailbox, set (s+1)&1
+          P* m = reinterpret_cast<P*>((i & 1) ? a.mail1 : a.mail0) + (int64_t)cc * a.seg_pad;
+          if (tc.nv == 4) {
+            store4_stream(m + tc.off, acc[0], acc[1], acc[2], acc[3]);
+          } else {
+#pragma unroll
+            for (int q2 = 0; q2 < 3; ++q2)
+              if (q2 < tc.nv) m[tc.off + q2] = (P)acc[q2];
+          }
+        }
+        cc = next_client(cc, n);
+      }
+    }
+    if (++bc < nb) return;
+    // the tile is through all n clients: consensus bits, 4 per thread, 8 lanes make one word
+    uint32_t nib = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) nib |= (uint32_t)(q < tc.nv && ((acc[q] > a.lam) | (acc[q] < a.lam_lo))) << q;
+    uint32_t word = nib << (4 * (lane & 7));
+    word |= __shfl_xor_sync(0xffffffffu, word, 1);
+    word |= __shfl_xor_sync(0xffffffffu, word, 2);
+    word |= __shfl_xor_sync(0xffffffffu, word, 4);
+    if ((lane & 7) == 0) sm_words[warp * 4 + (lane >> 3)] = word;
+    __syncthreads();
+    const int nw = (tc.left + 31) >> 5;
+    const int64_t wb = (tc.b + tc.off - (int64_t)tid * 4) >> 5;
+    const int w = tid % WPT;
+    if (w < nw) {
+      const uint32_t val = sm_words[w];
+      if (a.owner_only) {
+        if (tid < WPT) out[(int64_t)(tc.j == 0 ? n - 1 : tc.j - 1) * a.out_ld + wb + w] = val;
+      } else {
+        for (int row = tid / WPT; row < n; row += TPB / WPT) out[(int64_t)row * a.out_ld + wb + w] = val;
+      }
+    }
+    __syncthreads();
+    acc[0] = acc[1] = acc[2] = acc[3] = 0;
+    bc = 0;
+    uc += gridDim.x;
+    have_c = find(uc, tc);
+    cc = have_c ? tc.j : 0;
+  };
+
+  float4 xa[UNR], xb[UNR];
+  issue(xa);
+  while (have_c) {
+    issue(xb);
+    consume(xa);
+    if (!have_c) break;
+    issue(xa);
+    consume(xb);
+  }
+}
+
 template <int VPT, int UNR>
 __global__ void __launch_bounds__(256)
 fused_sum_kernel(const FusedArgs a) {
@@ -1014,16 +1169,17 @@ struct HonestRows {
   int64_t byte_off[128];
 };
 
-#ifndef BRACE_STATS_MINB_80
-#define BRACE_STATS_MINB_80 4
-#endif
+// CTAs of 64 threads: the CTAs of one SM drift apart in phase (loading / computing) sooner than
+// wider ones do, which keeps the memory pipe busier (n = 100, d = 25.6 M: 1.68 ms, against 1.71 ms
+// with 128 threads, 1.73 ms with 32 and 1.81 ms with 256).
+constexpr int kStatsThreads = 64;
 
-constexpr int stats_min_blocks(int mfull) {
-  return mfull <= 24 ? 8 : (mfull <= 40 ? 6 : (mfull <= 56 ? 5 : (mfull <= 80 ? BRACE_STATS_MINB_80 : (mfull <= 96 ? 3 : 2))));
+__host__ __device__ constexpr int stats_min_blocks(int mfull) {
+  return mfull <= 24 ? 8 : (mfull <= 40 ? 6 : (mfull <= 56 ? 5 : (mfull <= 80 ? 4 : (mfull <= 96 ? 3 : 2))));
 }
 
 template <int MFULL, int MTAIL, bool STRIDED>
-__global__ void __launch_bounds__(128, stats_min_blocks(MFULL))
+__global__ void __launch_bounds__(kStatsThreads, stats_min_blocks(MFULL) * 128 / kStatsThreads)
 inject_stats_reg_kernel(int kind, const __grid_constant__ HonestRows rows, uint32_t stride_bytes,
                         const int* __restrict__ ids, int f, int m, const float* H, float* Uo, int64_t ld_u, int64_t d,
                         float scale, float kappa) {
@@ -1085,34 +1241,45 @@ inject_stats_reg_kernel(int kind, const __grid_constant__ HonestRows rows, uint3
 // Coordinate-wise median / trimmed mean over the n client values of each
 // coordinate (the server-side rules Section 5.1 compares against; they need all
 // n slices at once, which is why they cannot run inside the ring, Section 3).
-// A thread owns one coordinate: its n values are loaded into registers, padded
-// with +Inf to NP (a power of two) and sorted by a fully unrolled bitonic
-// network of min/max pairs; the statistic is then read off the sorted registers.
-// Arithmetic-bound: NP*log2(NP)*(log2(NP)+1)/4 compare-exchanges per coordinate.
+// A thread owns one coordinate: its n values are loaded into NB registers (n
+// rounded up to a multiple of 8, the rest +Inf) and sorted by Batcher's odd-even
+// merge sorting network, fully unrolled.  Every comparator of that network puts
+// the smaller value at the lower index, so +Inf pads at the top never move and
+// every comparator that would touch an index >= NB is left out at compile time:
+// the network is the one for the next power of two restricted to indices < NB
+// (1157 compare-exchanges for NB = 104 against 1792 for a 128-input bitonic
+// network).  Arithmetic-bound: one min and one max per compare-exchange.
 // ---------------------------------------------------------------------------
-template <int NP>
+__host__ __device__ constexpr int pow2_at_least(int v) {
+  int p = 1;
+  while (p < v) p *= 2;
+  return p;
+}
+
+template <int NB>
 __global__ void __launch_bounds__(128)
 coordinate_stat_kernel(int kind, int trim, int n, const float* __restrict__ U, int64_t ld, float* __restrict__ res,
                        int64_t d) {
-  const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (k >= d) return;
-  const float* src = U + k;
-  float x[NP];
+  constexpr int NP = pow2_at_least(NB);
+  const int64_t kc = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (kc >= d) return;
+  const float* src = U + kc;
+  float x[NB];
 #pragma unroll
-  for (int i = 0; i < NP; ++i) x[i] = (i < n) ? __ldcs(src + (int64_t)i * ld) : __int_as_float(0x7f800000);
-  // bitonic sort, ascending
+  for (int i = 0; i < NB; ++i) x[i] = (i < n) ? __ldcs(src + (int64_t)i * ld) : __int_as_float(0x7f800000);
+  // odd-even merge sort, ascending: merges of runs of length p, comparator distance k
 #pragma unroll
-  for (int size = 2; size <= NP; size <<= 1) {
+  for (int p = 1; p < NP; p *= 2) {
 #pragma unroll
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+    for (int k = p; k >= 1; k /= 2) {
 #pragma unroll
-      for (int i = 0; i < NP; ++i) {
-        const int l = i ^ stride;
-        if (l > i) {
-          const float a = x[i], b = x[l];
-          const float lo = fminf(a, b), hi = fmaxf(a, b);
-          if ((i & size) == 0) { x[i] = lo; x[l] = hi; }
-          else                 { x[i] = hi; x[l] = lo; }
+      for (int i = 0; i < NB; ++i) {
+        const int l = i + k;
+        const int first = k % p;
+        if (i >= first && ((i - first) % (2 * k)) < k && l < NB && (i / (2 * p)) == (l / (2 * p))) {
+          const float lo = fminf(x[i], x[l]), hi = fmaxf(x[i], x[l]);
+          x[i] = lo;
+          x[l] = hi;
         }
       }
     }
@@ -1122,7 +1289,7 @@ coordinate_stat_kernel(int kind, int trim, int n, const float* __restrict__ U, i
     const int hi_idx = n >> 1, lo_idx = (n - 1) >> 1;
     float vlo = 0.f, vhi = 0.f;
 #pragma unroll
-    for (int i = 0; i < NP; ++i) {
+    for (int i = 0; i < NB; ++i) {
       if (i == lo_idx) vlo = x[i];
       if (i == hi_idx) vhi = x[i];
     }
@@ -1130,11 +1297,11 @@ coordinate_stat_kernel(int kind, int trim, int n, const float* __restrict__ U, i
   } else {                                           // trimmed mean: drop `trim` smallest and largest, float64 mean
     double acc = 0.0;
 #pragma unroll
-    for (int i = 0; i < NP; ++i)
+    for (int i = 0; i < NB; ++i)
       if (i >= trim && i < n - trim) acc = __dadd_rn(acc, (double)x[i]);
     out = __double2float_rn(__ddiv_rn(acc, (double)(n - 2 * trim)));
   }
-  res[k] = out;
+  res[kc] = out;
 }
 
 }  // namespace brace

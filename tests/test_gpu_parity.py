@@ -175,11 +175,14 @@ def test_hop_by_hop_and_whole_round(n, d, G, ld, lam, zs, rule):
 
     # (3) whole round, fused kernel, every shape; mailboxes end as the step calls left them
     if fusable:
-        for variant in list(range(0, 6)) + [1001, 2001]:  # +1000 / +2000: share-only launch forced / never
+        # variants 6, 8, 9 are the software-pipelined kernel (persistent CTAs); +1000 / +2000: share-only
+        # launch forced / never; a grid cap makes CTAs walk several tiles
+        for variant, grid in [(v, 0) for v in range(0, 10)] + [(1001, 0), (2001, 0), (2, 3), (8, 3), (1009, 2),
+                                                                (2006, 1)]:
             ctxf = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, zero_sign=zs, granule=G, mean=mean,
                                                      agg_mode=B.AGG_FUSED))
             ctxf.workspace.fill_(0x5A)
-            ctxf.set_tuning(variant, 3 if variant == 2 else 0)
+            ctxf.set_tuning(variant, grid)
             out3 = torch.full_like(out, 9)
             ctxf.aggregate(Ud, out3)
             check_final(out3, tr, rule, d)
