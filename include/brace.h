@@ -313,12 +313,10 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
                         int64_t* len, int32_t* segment, int32_t* entry_bytes);
 
 /* Expert knob for measurements: pick the fused kernel's shape.  fused_variant
- * 0 = library default; 1..5 and 7 = (float4 per thread per client, clients
+ * 0 = library default; 1..6 = (float4 per thread per client, clients
  * prefetched, threads per CTA) in {(1,8,256),(2,4,256),(1,4,256),(2,8,256),
- * (1,16,256)} and (1,8,128); 6, 8, 9 = the software-pipelined kernel with
- * persistent CTAs and (clients per batch, threads per CTA) in {(4,128),(8,128),
- * (8,256)}.  fused_grid = 0 launches one CTA per tile (pipelined kernel: as many
- * CTAs as stay resident), > 0 caps the grid (CTAs then loop over tiles).
+ * (1,16,256),(1,8,128)}.  fused_grid = 0 launches one CTA per tile, > 0 caps the
+ * grid (CTAs then loop over tiles).
  * Adding 10, 20 or 40 to fused_variant makes the share-reduce hop kernel process
  * 1, 2 or 4 float4 per thread (default: 4, fewer for short sub-vectors); adding
  * 100, 200 or 400 picks the staged statistics kernel with 1, 2 or 4 floats per
@@ -327,6 +325,8 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
  * (n*d >= 2^27) the fused kernel writes each sub-vector's bits to its owner's row
  * and one share-only launch spreads them to the other rows; adding 1000 forces
  * that at any size, adding 2000 makes the fused kernel write all n rows itself.
+ * A launch of only a few waves of CTAs uses narrower tiles so that its CTAs fill
+ * whole waves; adding 4000 keeps the full tile width.
  * Results do not depend on any of these. */
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid);
 

@@ -386,6 +386,7 @@ struct FusedArgs {
   int zs;
   int mean;
   int tiles_per_seg;
+  int tile_w;       // coordinates per tile (sign rules: may be narrower than the CTA covers)
   int64_t units;
   int owner_only;   // sign rules: write the consensus bits to the owner's row only (a share-only kernel follows)
 };
@@ -403,13 +404,32 @@ fused_sign_kernel(const FusedArgs a) {
   const float* __restrict__ U = a.U;
   uint32_t* __restrict__ out = reinterpret_cast<uint32_t*>(a.out);
 
+  // tile_w <= TILE coordinates of a tile are used (a multiple of 32): the host narrows the tiles of
+  // short launches so that the CTAs fill a whole number of waves
+  const int tile_w = a.tile_w;
+  const uint32_t tps = (uint32_t)a.tiles_per_seg;
+  const bool small = a.units < ((int64_t)1 << 31) && (int64_t)n * pt.Q < ((int64_t)1 << 31);
   for (int64_t u = blockIdx.x; u < a.units; u += gridDim.x) {
-    const int j = (int)(u / a.tiles_per_seg);
-    const int k = (int)(u % a.tiles_per_seg);
-    const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+    int j, k;
+    int64_t b, e;
+    if (small) {                                   // everything fits 32-bit divisions
+      j = (int)((uint32_t)u / tps);
+      k = (int)((uint32_t)u - (uint32_t)j * tps);
+      const uint32_t q = (uint32_t)pt.Q, un = (uint32_t)n;
+      b = pt.G * (int64_t)(((uint32_t)j * q) / un);
+      e = pt.G * (int64_t)(((uint32_t)(j + 1) * q) / un);
+      b = b < pt.d ? b : pt.d;
+      e = (j + 1 == n || e > pt.d) ? pt.d : e;
+    } else {
+      j = (int)(u / a.tiles_per_seg);
+      k = (int)(u % a.tiles_per_seg);
+      b = pt.begin(j);
+      e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+    }
     const int64_t L = e - b;
-    const int64_t t0 = (int64_t)k * TILE;
+    const int64_t t0 = (int64_t)k * tile_w;
     if (t0 >= L) continue;                         // uniform over the CTA
+    const int64_t tile_end = t0 + tile_w < L ? t0 + tile_w : L;   // first coordinate past this tile
 
     int64_t off[VPT];
     int nv[VPT];
@@ -417,7 +437,7 @@ fused_sign_kernel(const FusedArgs a) {
 #pragma unroll
     for (int v = 0; v < VPT; ++v) {
       off[v] = t0 + (int64_t)(v * TPB + tid) * 4;
-      const int64_t rem = L - off[v];
+      const int64_t rem = tile_end - off[v];
       nv[v] = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
       acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0;
     }
@@ -478,8 +498,7 @@ fused_sign_kernel(const FusedArgs a) {
       if ((lane & 7) == 0) sm_words[v * (TPB / 8) + warp * 4 + (lane >> 3)] = word;
     }
     __syncthreads();
-    const int64_t left = L - t0;
-    const int nw = left >= TILE ? WPT : (int)((left + 31) >> 5);
+    const int nw = (int)((tile_end - t0 + 31) >> 5);
     const int64_t wb = (b + t0) >> 5;
     const int w = tid % WPT;
     if (w < nw) {
@@ -491,161 +510,6 @@ fused_sign_kernel(const FusedArgs a) {
       }
     }
     __syncthreads();
-  }
-}
-
-// Software-pipelined form of the fused round for problems of a few L2 sizes or
-// less, where a launch is too short for the CTAs' load and compute phases to
-// drift apart on their own.  A persistent CTA walks its tiles (tile u, then
-// u + gridDim.x, ...) as one flat sequence of client batches; the loads of the
-// next batch -- of the same tile or of the CTA's next tile -- are issued before
-// the current batch is consumed, so every warp always has UNR loads in flight.
-// Tile width is TPB * 4 coordinates (one float4 per thread per client).  The
-// result and the two surviving mailbox states are those of fused_sign_kernel.
-template <typename P, int UNR, bool ZS, int TPB>
-__global__ void __launch_bounds__(TPB)
-fused_sign_pipe_kernel(const FusedArgs a) {
-  constexpr int TILE = TPB * 4;
-  constexpr int WPT = TPB / 8;                       // output words per tile
-  __shared__ uint32_t sm_words[WPT];
-  const Part pt = a.pt;
-  const int n = pt.n;
-  const int nb = (n + UNR - 1) / UNR;                // client batches per tile
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const float* __restrict__ U = a.U;
-  uint32_t* __restrict__ out = reinterpret_cast<uint32_t*>(a.out);
-  const uint32_t tps = (uint32_t)a.tiles_per_seg;
-  const bool small = a.units < ((int64_t)1 << 31) && (int64_t)n * pt.Q < ((int64_t)1 << 31);
-
-  struct Tile {
-    int64_t b;      // first coordinate of the sub-vector
-    int64_t off;    // this thread's first coordinate within the sub-vector
-    int j;          // sub-vector
-    int nv;         // valid coordinates of this thread's float4 (0..4)
-    int left;       // coordinates of the sub-vector from the tile's start on (capped at TILE)
-  };
-  // first non-empty tile at or after u in this CTA's sequence; false when the sequence is exhausted
-  auto find = [&](int64_t& u, Tile& t) -> bool {
-    for (; u < a.units; u += gridDim.x) {
-      int j, k;
-      int64_t b, e;
-      if (small) {                                   // 32-bit divisions
-        j = (int)((uint32_t)u / tps);
-        k = (int)((uint32_t)u - (uint32_t)j * tps);
-        const uint32_t q = (uint32_t)pt.Q, un = (uint32_t)n;
-        b = pt.G * (int64_t)(((uint32_t)j * q) / un);
-        e = pt.G * (int64_t)(((uint32_t)(j + 1) * q) / un);
-        b = b < pt.d ? b : pt.d;
-        e = (j + 1 == n || e > pt.d) ? pt.d : e;
-      } else {
-        j = (int)(u / tps);
-        k = (int)(u % tps);
-        b = pt.begin(j);
-        e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
-      }
-      const int64_t L = e - b, t0 = (int64_t)k * TILE;
-      if (t0 >= L) continue;
-      t.b = b;
-      t.j = j;
-      t.off = t0 + (int64_t)tid * 4;
-      const int64_t rem = L - t.off;
-      t.nv = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
-      t.left = (int)(L - t0 < TILE ? L - t0 : TILE);
-      return true;
-    }
-    return false;
-  };
-
-  // ---- loader state
-  int64_t ul = blockIdx.x;
-  Tile tl;
-  bool have_l = find(ul, tl);
-  int bl = 0, cl = have_l ? tl.j : 0;                // batch within the tile, client of the next load
-  // ---- consumer state
-  int64_t uc = ul;
-  Tile tc = tl;
-  bool have_c = have_l;
-  int bc = 0, cc = cl;
-  int acc[4] = {0, 0, 0, 0};
-
-  auto issue = [&](float4 (&x)[UNR]) {
-    if (!have_l) return;
-    const float* p = U + tl.b + tl.off;
-#pragma unroll
-    for (int q = 0; q < UNR; ++q) {
-      if (bl * UNR + q < n) {
-        x[q] = tl.nv > 0 ? ld_stream(p + (int64_t)cl * a.ld) : make_float4(0.f, 0.f, 0.f, 0.f);
-        cl = next_client(cl, n);
-      }
-    }
-    if (++bl == nb) {
-      bl = 0;
-      ul += gridDim.x;
-      have_l = find(ul, tl);
-      cl = have_l ? tl.j : 0;
-    }
-  };
-
-  auto consume = [&](float4 (&x)[UNR]) {
-#pragma unroll
-    for (int q = 0; q < UNR; ++q) {
-      const int i = bc * UNR + q;
-      if (i < n) {
-        acc[0] += sgn1<ZS>(x[q].x, a.zs);
-        acc[1] += sgn1<ZS>(x[q].y, a.zs);
-        acc[2] += sgn1<ZS>(x[q].z, a.zs);
-        acc[3] += sgn1<ZS>(x[q].w, a.zs);
-        if (i >= 1 && i >= n - 2) {                  // hop s = i-1 lands in client cc's mailbox, set (s+1)&1
-          P* m = reinterpret_cast<P*>((i & 1) ? a.mail1 : a.mail0) + (int64_t)cc * a.seg_pad;
-          if (tc.nv == 4) {
-            store4_stream(m + tc.off, acc[0], acc[1], acc[2], acc[3]);
-          } else {
-#pragma unroll
-            for (int q2 = 0; q2 < 3; ++q2)
-              if (q2 < tc.nv) m[tc.off + q2] = (P)acc[q2];
-          }
-        }
-        cc = next_client(cc, n);
-      }
-    }
-    if (++bc < nb) return;
-    // the tile is through all n clients: consensus bits, 4 per thread, 8 lanes make one word
-    uint32_t nib = 0;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) nib |= (uint32_t)(q < tc.nv && ((acc[q] > a.lam) | (acc[q] < a.lam_lo))) << q;
-    uint32_t word = nib << (4 * (lane & 7));
-    word |= __shfl_xor_sync(0xffffffffu, word, 1);
-    word |= __shfl_xor_sync(0xffffffffu, word, 2);
-    word |= __shfl_xor_sync(0xffffffffu, word, 4);
-    if ((lane & 7) == 0) sm_words[warp * 4 + (lane >> 3)] = word;
-    __syncthreads();
-    const int nw = (tc.left + 31) >> 5;
-    const int64_t wb = (tc.b + tc.off - (int64_t)tid * 4) >> 5;
-    const int w = tid % WPT;
-    if (w < nw) {
-      const uint32_t val = sm_words[w];
-      if (a.owner_only) {
-        if (tid < WPT) out[(int64_t)(tc.j == 0 ? n - 1 : tc.j - 1) * a.out_ld + wb + w] = val;
-      } else {
-        for (int row = tid / WPT; row < n; row += TPB / WPT) out[(int64_t)row * a.out_ld + wb + w] = val;
-      }
-    }
-    __syncthreads();
-    acc[0] = acc[1] = acc[2] = acc[3] = 0;
-    bc = 0;
-    uc += gridDim.x;
-    have_c = find(uc, tc);
-    cc = have_c ? tc.j : 0;
-  };
-
-  float4 xa[UNR], xb[UNR];
-  issue(xa);
-  while (have_c) {
-    issue(xb);
-    consume(xa);
-    if (!have_c) break;
-    issue(xa);
-    consume(xb);
   }
 }
 

@@ -1,12 +1,17 @@
 """Parity at the full sizes of the five workloads, in the launch configuration
-bench.py times (fused round, default tuning; injection in its default kernels).
+bench.py times (fused round, default tuning; injection in its default kernels,
+attacks 2 and 5 drawing inside the kernel).
 
-The oracle cannot run 2.5e9 elements in test time, so the comparison is on
-sampled coordinates it computes one by one (Eq. (1) per coordinate needs only
-that coordinate's column): the head and the ragged tail of the vector, both
-sides of sub-vector boundaries, and random coordinates.  Properties that hold
-at any size are checked on the whole result: every client's row is identical,
-padding bits are zero, the hop-by-hop path leaves the same bits and mailboxes."""
+Every bit is compared: the device matrices are streamed back in coordinate
+slabs, the oracle runs on each slab (Eq. (1) is per coordinate, so a slab is an
+independent problem) and is compared with every output word of client 0's row
+and with every owner's final sign-sums; the other clients' rows are compared
+with client 0's on the device.  A sampled comparison runs first as a fast
+pre-check.  Slabs are handed to a few host threads (numpy releases the GIL);
+each thread calls the oracle as it stands."""
+
+import concurrent.futures as cf
+import os
 
 import numpy as np
 import pytest
@@ -18,6 +23,8 @@ from paper_2501_17392_b200 import build as brace_build
 from paper_2501_17392_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
+REL_TOL = 1e-5
+THREADS = max(1, min(12, len(os.sched_getaffinity(0))))
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -41,81 +48,158 @@ def bits_at(row_words: torch.Tensor, idx: torch.Tensor) -> np.ndarray:
     return ((w >> (idx % 32)) & 1).cpu().numpy().astype(np.int8)
 
 
-def one_round(w, ctx, H, noise, unif, rnd):
-    d, n = w.d, w.n
-    idx_np = sample_coordinates(ctx, d, n, seed=rnd + n)
-    idx = torch.as_tensor(idx_np, device="cuda")
-    Hs = H[:, idx].cpu().numpy()
-    atk = B.make_attack(w.attack, scale=w.scale, sigma=w.sigma, kappa=w.kappa, prob=w.prob, noise=noise, uniform=unif)
-    ctx.inject_attack(atk, H, H)                       # in place, as a Byzantine client would
-    U = H
-    Us = U[:, idx].cpu().numpy()
-    exp_u = O.inject_attack(w.attack, Hs, list(range(w.f)), scale=w.scale, sigma=w.sigma, kappa=w.kappa, prob=w.prob,
-                            noise=None if noise is None else noise[:, idx].cpu().numpy(),
-                            uniform=None if unif is None else unif[:, idx].cpu().numpy())
-    rel = np.abs(Us - exp_u) / np.maximum(np.abs(exp_u), 1e-30)
-    assert rel.max() <= 1e-5
-    assert np.array_equal(Us.view(np.uint32), exp_u.view(np.uint32))
+def slab_width(n: int) -> int:
+    """Coordinates per slab: a multiple of 128, about 2e8 elements per slab at most."""
+    return int(max(1 << 18, min(1 << 22, (200_000_000 // n) // 128 * 128)))
 
-    out = ctx.new_output()
-    out.fill_(-1)
-    ctx.aggregate(U, out)
-    torch.cuda.synchronize()
+
+def owners_sign_sums(ctx: B.Brace, n: int) -> torch.Tensor:
+    """The d final sign-sums, gathered from the mailboxes of the sub-vectors' owners
+    (client j-1 owns sub-vector j) in coordinate order, on the device."""
+    parts = []
+    for j in range(n):
+        owner = (j - 1) % n
+        p, ln, seg, eb = ctx.debug_mailbox(owner, 0)
+        assert seg == j and eb == 1
+        off = p - ctx.workspace.data_ptr()
+        parts.append(ctx.workspace[off: off + ln].view(torch.int8))
+    return torch.cat(parts)
+
+
+def check_slab(w, lam, byz, U_slab, out_words, sums, start, atk_check):
+    """Oracle on one slab of all n rows against the result words and sign-sums of the same coordinates."""
+    width = U_slab.shape[1]
+    total = O.sign_sum_direct(U_slab)
+    assert np.array_equal(total.astype(np.int8), sums), f"sign-sums differ in slab at {start}"
+    pm1 = O.consensus_map(total, O.RULE_SIGN_CONSENSUS, lam, w.n)
+    exp_words = O.pack_bits_fast(pm1)
+    assert np.array_equal(exp_words, out_words), f"output words differ in slab at {start}"
+    if start == 0:                                    # the definition in one piece, once
+        assert np.array_equal(O.gar_direct(U_slab[:, :65536], lam), pm1[:65536])
+    if atk_check is None or not byz:
+        return
+    if w.attack in (O.ATTACK_SCALED_MEAN, O.ATTACK_MEAN_SHIFT):
+        # the honest rows of the injected matrix are the honest matrix (checked on the device)
+        exp = O.inject_attack(w.attack, U_slab, byz, scale=w.scale, kappa=w.kappa)
+        assert np.array_equal(exp[byz].view(np.uint32), U_slab[byz].view(np.uint32)), f"injected rows differ at {start}"
+    elif w.attack in (O.ATTACK_GAUSSIAN, O.ATTACK_SPARSE_NOISE):
+        seed, rnd = atk_check
+        noise, unif = O.attack_draws(w.attack, seed, rnd, byz, width, start=start)
+        exp = O.inject_attack(w.attack, U_slab, byz, sigma=w.sigma, prob=w.prob, noise=noise, uniform=unif)[byz]
+        got = U_slab[byz]
+        assert np.array_equal(got == 0, exp == 0), f"altered coordinates differ at {start}"
+        assert (np.abs(got.astype(np.float64) - exp) <= REL_TOL * np.abs(exp.astype(np.float64))).all()
+
+
+def full_compare(w, ctx, U, out, lam, byz, atk_check, draws_every=1):
+    """Every output word of row 0 and every final sign-sum against the oracle, slab by slab; rows 1..n-1
+    against row 0 on the device."""
+    n, d = w.n, w.d
     words = (d + 31) // 32
-    # any-size properties
     for c in range(1, n):
         assert torch.equal(out[c, :words], out[0, :words]), f"client {c} differs from client 0"
     if d % 32:
-        last = int(out[0, words - 1].item()) & 0xFFFFFFFF
-        assert last >> (d % 32) == 0, "padding bits must be zero"
-    # sampled coordinates against Eq. (1)
-    exp_bits = (O.gar_direct(exp_u, w.lam) > 0).astype(np.int8)
-    assert np.array_equal(bits_at(out[0], idx), exp_bits)
-    # the owners' final partial sign-sums at the sampled coordinates
-    S = O.sign_sum_direct(exp_u)
-    for j in sorted(set([0, 1, n // 2, n - 1])):
-        owner = (j - 1) % n
-        b, e = ctx.segment(j)
-        seg, box = ctx.mailbox_tensor(owner)
-        assert seg == j and box.numel() == e - b
-        sel = (idx_np >= b) & (idx_np < e)
-        assert np.array_equal(box.numpy()[idx_np[sel] - b].astype(np.int32), S[sel])
-    return out, U
+        assert (int(out[0, words - 1].item()) & 0xFFFFFFFF) >> (d % 32) == 0, "padding bits must be zero"
+    sums_dev = owners_sign_sums(ctx, n)
+    assert sums_dev.numel() == d
+    out0 = out[0, :words].cpu().numpy().view(np.uint32)
+    sums = sums_dev.cpu().numpy()
+    del sums_dev
+    S = slab_width(n)
+    starts = list(range(0, d, S))
+    stats_attack = w.attack in (O.ATTACK_SCALED_MEAN, O.ATTACK_MEAN_SHIFT)
+    with cf.ThreadPoolExecutor(max_workers=THREADS) as pool:
+        pending = []
+        for i, a in enumerate(starts):
+            b = min(d, a + S)
+            U_slab = U[:, a:b].cpu().numpy()
+            check = atk_check if (stats_attack or i % draws_every == 0 or i == len(starts) - 1) else None
+            pending.append(pool.submit(check_slab, w, lam, byz, U_slab, out0[a // 32: (b + 31) // 32], sums[a:b], a,
+                                       check))
+            while len(pending) > THREADS + 2:
+                pending.pop(0).result()
+        for fut in pending:
+            fut.result()
+
+
+def sampled_precheck(w, ctx, U, out, lam):
+    idx_np = sample_coordinates(ctx, w.d, w.n, seed=w.n)
+    idx = torch.as_tensor(idx_np, device="cuda")
+    cols = U[:, idx].cpu().numpy()
+    assert np.array_equal(bits_at(out[0], idx), (O.gar_direct(cols, lam) > 0).astype(np.int8))
 
 
 @pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
 def test_full_size_workload(name):
     w = W.WORKLOADS[name]
-    ctx = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam, agg_mode=B.AGG_FUSED))
-    H = torch.zeros((w.n, w.ld), dtype=torch.float32, device="cuda")
-    out = U = None
+    n, f, d = w.n, w.f, w.d
+    ctx = B.Brace(n, f, d, B.default_params(lam=w.lam, agg_mode=B.AGG_FUSED))
+    H = torch.zeros((n, w.ld), dtype=torch.float32, device="cuda")
+    U = torch.empty_like(H)
+    out = ctx.new_output()
+    byz = list(range(f))
+    generated = w.attack in (W.ATTACK_GAUSSIAN, W.ATTACK_SPARSE_NOISE)
+    seed = W.BASE_SEED + n
     for rnd in range(w.rounds):
         W.honest_updates(w, rnd, device="cuda", out=H)
-        noise, unif = W.attack_draws(w, rnd, device="cuda")
-        out, U = one_round(w, ctx, H, noise, unif, rnd)
-        del noise, unif
+        U.copy_(H)
+        atk = B.make_attack(w.attack, scale=w.scale, sigma=w.sigma, kappa=w.kappa, prob=w.prob,
+                            seed=seed if generated else None, round_idx=rnd)
+        ctx.inject_attack(atk, H, U)
+        assert torch.equal(U[f:], H[f:]), "honest rows must not change"
+        assert torch.equal(U[:, d:], H[:, d:]), "row padding must not change"
+        out.fill_(-1)
+        ctx.aggregate(U, out)
+        torch.cuda.synchronize()
+        sampled_precheck(w, ctx, U, out, w.lam)
+        full_compare(w, ctx, U, out, w.lam, byz, (seed, rnd), draws_every=4 if name == "cfg5" else 1)
     # the hop-by-hop path on the same (last) inputs: same bits, same surviving mailboxes
-    ctx_s = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam, agg_mode=B.AGG_STEPWISE))
+    del H
+    torch.cuda.empty_cache()
+    ctx_s = B.Brace(n, f, d, B.default_params(lam=w.lam, agg_mode=B.AGG_STEPWISE))
     out_s = ctx_s.new_output()
     ctx_s.aggregate(U, out_s)
     torch.cuda.synchronize()
-    words = (w.d + 31) // 32
+    words = (d + 31) // 32
     assert torch.equal(out_s[:, :words], out[:, :words])
-    for c in sorted(set([0, 1, w.n // 2, w.n - 1])):
+    for c in range(n):
         for hb in (0, 1):
-            sa, a = ctx.mailbox_tensor(c, hb)
-            sb, b = ctx_s.mailbox_tensor(c, hb)
-            assert sa == sb and torch.equal(a, b)
+            pa, la, sa, _ = ctx.debug_mailbox(c, hb)
+            pb, lb, sb, _ = ctx_s.debug_mailbox(c, hb)
+            assert sa == sb and la == lb
+            oa, ob = pa - ctx.workspace.data_ptr(), pb - ctx_s.workspace.data_ptr()
+            assert torch.equal(ctx.workspace[oa: oa + la], ctx_s.workspace[ob: ob + lb])
     ctx.close()
     ctx_s.close()
-    del H
+    del U, out, out_s
     torch.cuda.empty_cache()
 
 
+def test_full_size_cfg1_with_its_attack():
+    """cfg1 at its real size (small enough for the oracle's hop-by-hop procedure in full)."""
+    w = W.WORKLOADS["cfg1"]
+    H = W.honest_updates(w, 0, device="cuda")
+    U = H.clone()
+    ctx = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam, agg_mode=B.AGG_FUSED))
+    ctx.inject_attack(B.make_attack(w.attack, scale=w.scale), H, U)
+    out = ctx.new_output()
+    ctx.aggregate(U, out)
+    torch.cuda.synchronize()
+    exp_u = O.inject_attack(w.attack, H.cpu().numpy()[:, :w.d], list(range(w.f)), scale=w.scale)
+    assert np.array_equal(U.cpu().numpy()[:, :w.d].view(np.uint32), exp_u.view(np.uint32))
+    tr = O.ring_round(exp_u, lam=w.lam, keep_states=False)
+    words = (w.d + 31) // 32
+    got = out[:, :words].cpu().numpy().view(np.uint32)
+    for c in range(w.n):
+        assert np.array_equal(got[c], O.pack_bits_fast(tr.outputs[c]))
+    full_compare(w, ctx, U, out, w.lam, list(range(w.f)), None)
+    ctx.close()
+
+
 def test_vector_longer_than_2_to_31():
-    """Two clients, d just above 2^31: every in-row offset needs 64-bit arithmetic.
-    Sampled coordinates (head, the 2^31 crossing, sub-vector boundary, tail, random) against Eq. (1),
-    both round modes, plus the attack and model-update kernels at the far end of the rows."""
+    """Two clients, d just above 2^31: every in-row offset needs 64-bit arithmetic.  Every output
+    word against Eq. (1), both round modes, plus the attack and model-update kernels at the far end of
+    the rows."""
     n, d = 2, (1 << 31) + 4_099
     ld = W.round_up(d, 128)
     free, _ = torch.cuda.mem_get_info()
@@ -125,6 +209,8 @@ def test_vector_longer_than_2_to_31():
     g = torch.Generator(device="cuda").manual_seed(99)
     for i in range(n):
         U[i].normal_(generator=g)
+    U[:, d:].zero_()
+    w = W.Workload("long", n, 1, d, 1, "gauss", W.ATTACK_SCALE_OWN, scale=-10.0)
     ctx = B.Brace(n, 1, d, B.default_params(lam=0.0, agg_mode=B.AGG_FUSED))
     rng = np.random.default_rng(5)
     b1, e1 = ctx.segment(1)
@@ -143,10 +229,9 @@ def test_vector_longer_than_2_to_31():
     ctx.aggregate(U, out)
     torch.cuda.synchronize()
     words = (d + 31) // 32
-    assert torch.equal(out[1, :words], out[0, :words])
     exp_bits = (O.gar_direct(exp_u, 0.0) > 0).astype(np.int8)
     assert np.array_equal(bits_at(out[0], idx), exp_bits)
-    assert (int(out[0, words - 1].item()) & 0xFFFFFFFF) >> (d % 32) == 0
+    full_compare(w, ctx, U, out, 0.0, [0], None)
     ctx_s = B.Brace(n, 1, d, B.default_params(lam=0.0, agg_mode=B.AGG_STEPWISE))
     out_s = ctx_s.new_output()
     ctx_s.aggregate(U, out_s)
@@ -165,8 +250,9 @@ def test_vector_longer_than_2_to_31():
 
 
 def test_full_size_sum_rule_cfg2():
-    """Plain ring-all-reduce at cfg2's size: fused and hop-by-hop give the same
-    float32 bits, sampled coordinates match the oracle's ring-order float32 sum."""
+    """Plain ring-all-reduce at cfg2's size: fused and hop-by-hop give the same float32 bits, and every
+    coordinate matches the float32 ring-order sum (sub-vector j is reduced starting at client j) and the
+    oracle's float64 sum within tolerance."""
     w = W.WORKLOADS["cfg2"]
     H = W.honest_updates(w, 0, device="cuda")
     outs = []
@@ -181,19 +267,13 @@ def test_full_size_sum_rule_cfg2():
     assert torch.equal(outs[0][:, :w.d].view(torch.int32), outs[1][:, :w.d].view(torch.int32))
     for c in range(1, w.n):
         assert torch.equal(outs[0][c, :w.d].view(torch.int32), outs[0][0, :w.d].view(torch.int32))
-    rng = np.random.default_rng(2)
-    idx = np.unique(np.concatenate([np.arange(0, 512), np.arange(w.d - 512, w.d), rng.integers(0, w.d, 4096)]))
-    Hs = H[:, torch.as_tensor(idx, device="cuda")].cpu().numpy()
-    got = outs[0][0, torch.as_tensor(idx, device="cuda")].cpu().numpy()
-    # sub-vector j is reduced starting at client j: same float32 add order, coordinate by coordinate
-    seg_of = np.searchsorted(np.array([b for b, _ in bounds] + [w.d]), idx, side="right") - 1
-    exp = np.empty(idx.size, dtype=np.float32)
-    for t, (k, j) in enumerate(zip(idx, seg_of)):
-        acc = Hs[j, t]
+    Hh = H.cpu().numpy()[:, :w.d]
+    got = outs[0][0, :w.d].cpu().numpy()
+    for j, (b, e) in enumerate(bounds):
+        acc = Hh[j, b:e].copy()
         for i in range(1, w.n):
-            acc = np.float32(acc + Hs[(j + i) % w.n, t])
-        exp[t] = acc
-    assert np.array_equal(got.view(np.uint32), exp.view(np.uint32))
-    ref = O.sum_direct_f64(Hs)
-    scale = np.abs(Hs.astype(np.float64)).sum(0)
+            acc = (acc + Hh[(j + i) % w.n, b:e]).astype(np.float32)     # float32 adds, ring order
+        assert np.array_equal(got[b:e].view(np.uint32), acc.view(np.uint32)), f"sub-vector {j}"
+    ref = O.sum_direct_f64(Hh)
+    scale = np.abs(Hh.astype(np.float64)).sum(0)
     assert (np.abs(got.astype(np.float64) - ref) <= 1e-5 * np.maximum(np.abs(ref), scale)).all()

@@ -175,10 +175,10 @@ def test_hop_by_hop_and_whole_round(n, d, G, ld, lam, zs, rule):
 
     # (3) whole round, fused kernel, every shape; mailboxes end as the step calls left them
     if fusable:
-        # variants 6, 8, 9 are the software-pipelined kernel (persistent CTAs); +1000 / +2000: share-only
-        # launch forced / never; a grid cap makes CTAs walk several tiles
-        for variant, grid in [(v, 0) for v in range(0, 10)] + [(1001, 0), (2001, 0), (2, 3), (8, 3), (1009, 2),
-                                                                (2006, 1)]:
+        # +1000 / +2000: share-only launch forced / never; +4000: tiles keep their full width; a grid cap
+        # makes CTAs walk several tiles
+        for variant, grid in [(v, 0) for v in range(0, 7)] + [(1001, 0), (2001, 0), (4001, 0), (5006, 0), (2, 3),
+                                                               (6, 2)]:
             ctxf = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, zero_sign=zs, granule=G, mean=mean,
                                                      agg_mode=B.AGG_FUSED))
             ctxf.workspace.fill_(0x5A)
@@ -533,6 +533,41 @@ def test_step_order_and_argument_errors():
     assert ctx.last_cuda_error() == 0
     ctx.close()
     ctx2.close()
+
+
+@pytest.mark.parametrize("n,d,zs", [(8, 700_001, 0), (3, 1_000_003, 1), (20, 1_663_370, 0), (50, 640_000, -1)])
+def test_fused_round_with_narrowed_tiles(n, d, zs):
+    """Launches of a few waves of CTAs get tiles narrower than a CTA covers (so that the CTAs fill whole
+    waves): same bits as Eq. (1), same surviving mailboxes as the hop-by-hop round, and as with full-width
+    tiles; an int16-partial case rides along."""
+    ld = W.round_up(d, 128)
+    g = torch.Generator(device="cuda").manual_seed(n * 1000 + 7)
+    U = torch.zeros((n, ld), dtype=torch.float32, device="cuda")
+    U[:, :d].normal_(generator=g)
+    U[:, :d][torch.rand((n, d), device="cuda", generator=g) < 0.05] = 0.0
+    lam = float(n // 7)
+    exp = O.pack_bits_fast(O.gar_direct(U.cpu().numpy()[:, :d], lam, zs))
+    words = (d + 31) // 32
+    ctx_s = B.Brace(n, 0, d, B.default_params(lam=lam, zero_sign=zs, agg_mode=B.AGG_STEPWISE))
+    out_s = ctx_s.new_output()
+    ctx_s.aggregate(U, out_s)
+    boxes_s = final_mailboxes(ctx_s)
+    for variant in (0, 4000, 6, 2):
+        ctx = B.Brace(n, 0, d, B.default_params(lam=lam, zero_sign=zs, agg_mode=B.AGG_FUSED))
+        ctx.workspace.fill_(0x33)
+        ctx.set_tuning(variant, 0)
+        out = torch.full_like(out_s, 5)
+        ctx.aggregate(U, out)
+        got = out[:, :words].cpu().numpy().view(np.uint32)
+        for c in range(n):
+            assert np.array_equal(got[c], exp), (variant, c)
+        boxes = final_mailboxes(ctx)
+        for hb in range(len(boxes_s)):
+            for c in range(n):
+                assert boxes[hb][c][0] == boxes_s[hb][c][0]
+                assert torch.equal(boxes[hb][c][1], boxes_s[hb][c][1]), (variant, hb, c)
+        ctx.close()
+    ctx_s.close()
 
 
 # ------------------------------------------------------------------ attack injection + whole pipeline

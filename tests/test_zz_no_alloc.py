@@ -4,18 +4,22 @@ Some users of this library run where device memory cannot be obtained at the
 moment they aggregate: inside a host application whose own allocator has taken
 all of HBM, or under a memory budget frozen at start-up.  They cannot provide
 the mailbox workspace `brace_init` wants, so the library carries a fixed
-scratch array of its own for them.  This test calls that entry point through
+scratch array of its own for them.  These tests call that entry point through
 the C ABI twice in a row (different inputs, the second call finding the first
-one's leftovers in the shared scratch) and requires the same bits as the
-ordinary `brace_aggregate` path, which the other GPU tests pin to the oracle.
-It lives in a file that sorts last so that a run stopping at the first failure
-has already been through every other test; it also passes on its own in a
-fresh process (it builds and loads the library itself).
+one's leftovers in the shared scratch) and require the bits the CPU oracle
+computes from the paper's definition -- the same expectation the ordinary
+`brace_aggregate` path is held to -- plus agreement with that path, and that the
+amount of free device memory is the same after the calls as before them.
+The file sorts last so that a run stopping at the first failure has already
+been through every other test; it also passes on its own in a fresh process (it
+builds and loads the library itself).
 """
 
+import numpy as np
 import pytest
 import torch
 
+from oracle import brace_oracle as O
 from paper_2501_17392_b200 import brace as B
 from paper_2501_17392_b200 import build as brace_build
 from paper_2501_17392_b200 import workloads as W
@@ -29,7 +33,7 @@ def _built():
     assert torch.cuda.is_available(), "this test needs a CUDA device"
 
 
-def _reference_round(n, d, params, U):
+def _workspace_round(n, d, params, U):
     ctx = B.Brace(n, 0, d, params)
     out = ctx.new_output()
     ctx.aggregate(U, out)
@@ -38,21 +42,78 @@ def _reference_round(n, d, params, U):
     return out
 
 
+def _new_output(n, d, rule):
+    if rule == B.RULE_SUM:
+        return torch.full((n, W.round_up(d, 4)), 7.0, dtype=torch.float32, device="cuda")
+    return torch.full((n, W.round_up((d + 31) // 32, 4)), 7, dtype=torch.int32, device="cuda")
+
+
 @pytest.mark.parametrize("rule", [B.RULE_SIGN_CONSENSUS, B.RULE_SUM])
-def test_static_scratch_round_matches_workspace_round_twice(rule):
+def test_static_scratch_round_matches_oracle_twice(rule):
     w = W.scaled(W.WORKLOADS["cfg2"], 300_001)            # 20 clients, several tiles, ragged tail
     params = B.default_params(rule=rule, lam=w.lam, agg_mode=B.AGG_FUSED)
+    inputs = [W.honest_updates(w, round_idx=call, device="cuda") for call in range(2)]
+    outs = [_new_output(w.n, w.d, rule) for _ in range(2)]
+    pristine = outs[0].clone()
+    B.aggregate_static(w.n, w.d, params, inputs[0], outs[0])      # first call on the device (loads the kernel)
+    torch.cuda.synchronize()
+    outs[0].copy_(pristine)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
     for call in range(2):                                  # two calls in a row share the scratch
-        U = W.honest_updates(w, round_idx=call, device="cuda")
-        expected = _reference_round(w.n, w.d, params, U)
-        out = torch.full_like(expected, 7)
-        B.aggregate_static(w.n, w.d, params, U, out)
-        torch.cuda.synchronize()
-        # bit-for-bit: integer work for the sign rule, same float32 add order for the sum rule;
+        B.aggregate_static(w.n, w.d, params, inputs[call], outs[call])
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "the entry point must not obtain device memory"
+    used = w.d if rule == B.RULE_SUM else (w.d + 31) // 32
+    for call in range(2):
+        Uh = inputs[call].cpu().numpy()[:, :w.d]
+        tr = O.ring_round(Uh, rule=O.RULE_SUM if rule == B.RULE_SUM else O.RULE_SIGN_CONSENSUS, lam=w.lam,
+                          keep_states=False)
+        got = outs[call].cpu().numpy()
+        for c in range(w.n):
+            if rule == B.RULE_SUM:        # float32 adds in ring order: the oracle's float32 trace, bit for bit
+                assert np.array_equal(got[c, :used].view(np.uint32), tr.outputs[c].view(np.uint32)), f"call {call}"
+            else:                         # integer work: the packed bits of Eq. (1)
+                assert np.array_equal(got[c, :used].view(np.uint32), O.pack_bits_fast(tr.outputs[c])), f"call {call}"
+        if rule != B.RULE_SUM:
+            assert np.array_equal(tr.outputs[0], O.gar_direct(Uh, w.lam))
+        # and the same bits as the round that uses a caller workspace
+        expected = _workspace_round(w.n, w.d, params, inputs[call])
+        assert torch.equal(outs[call].view(torch.int32)[:, :used], expected.view(torch.int32)[:, :used])
         # columns past the result (row padding) belong to the caller and stay as they were
-        used = w.d if rule == B.RULE_SUM else (w.d + 31) // 32
-        assert torch.equal(out.view(torch.int32)[:, :used], expected.view(torch.int32)[:, :used]), f"call {call}"
-        assert (out.view(torch.int32)[:, used:] == torch.full_like(expected, 7).view(torch.int32)[:, used:]).all()
+        assert torch.equal(outs[call].view(torch.int32)[:, used:], pristine.view(torch.int32)[:, used:])
+
+
+def test_static_scratch_large_problem_owner_rows_then_share_only():
+    """n * d >= 2^27 inside the 8 MiB limit: the fused kernel writes each sub-vector's bits to its owner's
+    row and a share-only launch spreads them; checked against Eq. (1) on every coordinate, twice."""
+    n, d = 100, 4_000_000
+    ld = W.round_up(d, 128)
+    params = B.default_params(lam=5.0, agg_mode=B.AGG_FUSED)
+    assert 2 * n * W.round_up(d // n, 128) <= B.STATIC_SCRATCH_BYTES
+    g = torch.Generator(device="cuda").manual_seed(2024)
+    U = torch.zeros((n, ld), dtype=torch.float32, device="cuda")
+    out = torch.zeros((n, W.round_up((d + 31) // 32, 4)), dtype=torch.int32, device="cuda")
+    B.aggregate_static(n, d, params, U, out)
+    torch.cuda.synchronize()
+    words = (d + 31) // 32
+    for call in range(2):
+        for i in range(n):
+            U[i, :d].normal_(0.02 * (call + 1), 1.0, generator=g)
+        out.fill_(-1)
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
+        B.aggregate_static(n, d, params, U, out)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
+        for c in range(1, n):
+            assert torch.equal(out[c, :words], out[0, :words])
+        got = out[0, :words].cpu().numpy().view(np.uint32)
+        step = 1_000_000
+        for a in range(0, d, step):
+            exp = O.pack_bits_fast(O.gar_direct(U[:, a: a + step].cpu().numpy(), 5.0))
+            assert np.array_equal(got[a // 32: (a + step) // 32], exp), f"call {call}, coordinates from {a}"
 
 
 def test_static_scratch_rejects_oversize_and_bad_layout():
@@ -68,3 +129,4 @@ def test_static_scratch_rejects_oversize_and_bad_layout():
     assert B.aggregate_static_status(4, 1024, B.default_params(granule=32), U, out) == B.ERR_UNSUPPORTED
     assert B.aggregate_static_status(4, 1024, p, U, out) == B.OK
     torch.cuda.synchronize()
+    assert B.lib().brace_last_cuda_error(None) == 0        # no CUDA failure recorded by the context-free calls
