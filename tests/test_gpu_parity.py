@@ -539,7 +539,7 @@ def test_step_order_and_argument_errors():
 def test_fused_round_with_narrowed_tiles(n, d, zs):
     """Launches of a few waves of CTAs get tiles narrower than a CTA covers (so that the CTAs fill whole
     waves): same bits as Eq. (1), same surviving mailboxes as the hop-by-hop round, and as with full-width
-    tiles; an int16-partial case rides along."""
+    tiles."""
     ld = W.round_up(d, 128)
     g = torch.Generator(device="cuda").manual_seed(n * 1000 + 7)
     U = torch.zeros((n, ld), dtype=torch.float32, device="cuda")
