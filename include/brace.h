@@ -325,8 +325,6 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
  * (n*d >= 2^27) the fused kernel writes each sub-vector's bits to its owner's row
  * and one share-only launch spreads them to the other rows; adding 1000 forces
  * that at any size, adding 2000 makes the fused kernel write all n rows itself.
- * A launch of only a few waves of CTAs uses narrower tiles so that its CTAs fill
- * whole waves; adding 4000 keeps the full tile width.
  * Results do not depend on any of these. */
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid);
 

@@ -60,7 +60,6 @@ struct brace_ctx {
   int step_vpt = 0;
   int spread_mode = 0;   // 0/1 = owner row + share-only launch when the layout allows, 2 = fused kernel writes all rows
   int stats_vw = 0;
-  int balance_waves = 1; // fused sign kernel: narrow the tiles of short launches to fill whole waves
   int stats_table = 0;   // 1 = statistics kernel addresses rows through the offset table even when they are consecutive
 };
 
@@ -279,30 +278,10 @@ bool fused_layout_ok(const brace_ctx* ctx, const float* U, int64_t ld, const voi
   return true;
 }
 
-// Tiles per sub-vector and their width.  `slots` > 0 (sign rules) is the number of CTAs the device
-// holds at once: a launch of only a few waves gets narrower tiles (a multiple of 32 coordinates, so
-// that tiles still start on output-word and 16-byte boundaries) chosen so that the CTAs fill a whole
-// number of waves -- otherwise the last, partly filled wave leaves SMs idle for a CTA's lifetime.
-void fused_geometry(const brace_ctx* ctx, FusedArgs& a, int64_t tile, int64_t slots) {
-  int64_t tps = (ctx->seg_max + tile - 1) / tile;
-  if (tps < 1) tps = 1;
-  int64_t width = tile;
-  const int64_t units = tps * ctx->n;
-  if (slots > 0 && ctx->balance_waves && units > slots && units < 12 * slots) {
-    const int64_t waves = (units + slots - 1) / slots;
-    const int64_t want = waves * slots / ctx->n;                 // tiles per sub-vector that fill the waves
-    if (want > tps) {
-      int64_t w = ((ctx->seg_max + want - 1) / want + 31) / 32 * 32;
-      if (w < 128) w = 128;
-      if (w < tile) {
-        width = w;
-        tps = (ctx->seg_max + width - 1) / width;
-      }
-    }
-  }
-  a.tiles_per_seg = (int)tps;
-  a.tile_w = (int)width;
-  a.units = tps * ctx->n;
+void fused_geometry(const brace_ctx* ctx, FusedArgs& a, int64_t tile) {
+  a.tiles_per_seg = (int)((ctx->seg_max + tile - 1) / tile);
+  if (a.tiles_per_seg < 1) a.tiles_per_seg = 1;
+  a.units = (int64_t)a.tiles_per_seg * ctx->n;
 }
 
 int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t out_ld, cudaStream_t st) {
@@ -338,7 +317,7 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
   };
 #define BRACE_FUSED_SIGN(VPT, UNR, TPB)                                                         \
   do {                                                                                          \
-    fused_geometry(ctx, a, (int64_t)TPB * 4 * VPT, (int64_t)ctx->sm_count * (1024 / TPB));      \
+    fused_geometry(ctx, a, (int64_t)TPB * 4 * VPT);                                             \
     const unsigned g = grid_for(a.units);                                                       \
     if (ctx->entry_bytes == 1) {                                                                \
       if (zs) fused_sign_kernel<int8_t, VPT, UNR, true, TPB><<<g, TPB, 0, st>>>(a);             \
@@ -350,7 +329,7 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
   } while (0)
 #define BRACE_FUSED_SUM(VPT, UNR)                                                               \
   do {                                                                                          \
-    fused_geometry(ctx, a, (int64_t)256 * 4 * VPT, 0);                                          \
+    fused_geometry(ctx, a, (int64_t)256 * 4 * VPT);                                             \
     const unsigned g = grid_for(a.units);                                                       \
     fused_sum_kernel<VPT, UNR><<<g, 256, 0, st>>>(a);                                           \
   } while (0)
@@ -734,10 +713,7 @@ int brace_last_cuda_error(const brace_ctx* ctx) { return ctx ? ctx->last_cuda : 
 
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid) {
   if (!ctx || fused_variant < 0 || fused_grid < 0) return BRACE_ERR_INVALID_ARG;
-  // thousands digit: 1 = always spread with a share-only launch, 2 = never; +4 = tiles keep their full width
-  const int thousands = fused_variant / 1000;
-  if (thousands > 6) return BRACE_ERR_INVALID_ARG;
-  const int spread_code = thousands & 3;
+  const int spread_code = fused_variant / 1000;  // thousands digit: 1 = always spread with a share-only launch, 2 = never
   fused_variant %= 1000;
   const int stats_code = fused_variant / 100;    // hundreds digit: floats per thread of the statistics kernel
   const int step_code = (fused_variant / 10) % 10;   // tens digit: float4 per thread of the hop kernel
@@ -747,7 +723,6 @@ int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid) 
     return BRACE_ERR_INVALID_ARG;
   if (spread_code < 0 || spread_code > 2) return BRACE_ERR_INVALID_ARG;
   ctx->spread_mode = spread_code;
-  ctx->balance_waves = (thousands & 4) ? 0 : 1;
   ctx->step_vpt = step_code;
   ctx->stats_vw = stats_code == 8 ? 0 : stats_code;
   ctx->stats_table = stats_code == 8 ? 1 : 0;

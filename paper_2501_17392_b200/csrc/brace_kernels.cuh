@@ -386,7 +386,6 @@ struct FusedArgs {
   int zs;
   int mean;
   int tiles_per_seg;
-  int tile_w;       // coordinates per tile (sign rules: may be narrower than the CTA covers)
   int64_t units;
   int owner_only;   // sign rules: write the consensus bits to the owner's row only (a share-only kernel follows)
 };
@@ -404,32 +403,13 @@ fused_sign_kernel(const FusedArgs a) {
   const float* __restrict__ U = a.U;
   uint32_t* __restrict__ out = reinterpret_cast<uint32_t*>(a.out);
 
-  // tile_w <= TILE coordinates of a tile are used (a multiple of 32): the host narrows the tiles of
-  // short launches so that the CTAs fill a whole number of waves
-  const int tile_w = a.tile_w;
-  const uint32_t tps = (uint32_t)a.tiles_per_seg;
-  const bool small = a.units < ((int64_t)1 << 31) && (int64_t)n * pt.Q < ((int64_t)1 << 31);
   for (int64_t u = blockIdx.x; u < a.units; u += gridDim.x) {
-    int j, k;
-    int64_t b, e;
-    if (small) {                                   // everything fits 32-bit divisions
-      j = (int)((uint32_t)u / tps);
-      k = (int)((uint32_t)u - (uint32_t)j * tps);
-      const uint32_t q = (uint32_t)pt.Q, un = (uint32_t)n;
-      b = pt.G * (int64_t)(((uint32_t)j * q) / un);
-      e = pt.G * (int64_t)(((uint32_t)(j + 1) * q) / un);
-      b = b < pt.d ? b : pt.d;
-      e = (j + 1 == n || e > pt.d) ? pt.d : e;
-    } else {
-      j = (int)(u / a.tiles_per_seg);
-      k = (int)(u % a.tiles_per_seg);
-      b = pt.begin(j);
-      e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
-    }
+    const int j = (int)(u / a.tiles_per_seg);
+    const int k = (int)(u % a.tiles_per_seg);
+    const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
     const int64_t L = e - b;
-    const int64_t t0 = (int64_t)k * tile_w;
+    const int64_t t0 = (int64_t)k * TILE;
     if (t0 >= L) continue;                         // uniform over the CTA
-    const int64_t tile_end = t0 + tile_w < L ? t0 + tile_w : L;   // first coordinate past this tile
 
     int64_t off[VPT];
     int nv[VPT];
@@ -437,7 +417,7 @@ fused_sign_kernel(const FusedArgs a) {
 #pragma unroll
     for (int v = 0; v < VPT; ++v) {
       off[v] = t0 + (int64_t)(v * TPB + tid) * 4;
-      const int64_t rem = tile_end - off[v];
+      const int64_t rem = L - off[v];
       nv[v] = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
       acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0;
     }
@@ -498,7 +478,8 @@ fused_sign_kernel(const FusedArgs a) {
       if ((lane & 7) == 0) sm_words[v * (TPB / 8) + warp * 4 + (lane >> 3)] = word;
     }
     __syncthreads();
-    const int nw = (int)((tile_end - t0 + 31) >> 5);
+    const int64_t left = L - t0;
+    const int nw = left >= TILE ? WPT : (int)((left + 31) >> 5);
     const int64_t wb = (b + t0) >> 5;
     const int w = tid % WPT;
     if (w < nw) {

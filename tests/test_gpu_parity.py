@@ -175,10 +175,8 @@ def test_hop_by_hop_and_whole_round(n, d, G, ld, lam, zs, rule):
 
     # (3) whole round, fused kernel, every shape; mailboxes end as the step calls left them
     if fusable:
-        # +1000 / +2000: share-only launch forced / never; +4000: tiles keep their full width; a grid cap
-        # makes CTAs walk several tiles
-        for variant, grid in [(v, 0) for v in range(0, 7)] + [(1001, 0), (2001, 0), (4001, 0), (5006, 0), (2, 3),
-                                                               (6, 2)]:
+        # +1000 / +2000: share-only launch forced / never; a grid cap makes CTAs walk several tiles
+        for variant, grid in [(v, 0) for v in range(0, 7)] + [(1001, 0), (2001, 0), (1006, 0), (2, 3), (6, 2)]:
             ctxf = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, zero_sign=zs, granule=G, mean=mean,
                                                      agg_mode=B.AGG_FUSED))
             ctxf.workspace.fill_(0x5A)
@@ -536,10 +534,9 @@ def test_step_order_and_argument_errors():
 
 
 @pytest.mark.parametrize("n,d,zs", [(8, 700_001, 0), (3, 1_000_003, 1), (20, 1_663_370, 0), (50, 640_000, -1)])
-def test_fused_round_with_narrowed_tiles(n, d, zs):
-    """Launches of a few waves of CTAs get tiles narrower than a CTA covers (so that the CTAs fill whole
-    waves): same bits as Eq. (1), same surviving mailboxes as the hop-by-hop round, and as with full-width
-    tiles."""
+def test_fused_round_medium_sizes(n, d, zs):
+    """Launches of a few waves of CTAs (between the tiny parity cases and the full-size workloads): same
+    bits as Eq. (1), same surviving mailboxes as the hop-by-hop round, several kernel shapes."""
     ld = W.round_up(d, 128)
     g = torch.Generator(device="cuda").manual_seed(n * 1000 + 7)
     U = torch.zeros((n, ld), dtype=torch.float32, device="cuda")
@@ -552,7 +549,7 @@ def test_fused_round_with_narrowed_tiles(n, d, zs):
     out_s = ctx_s.new_output()
     ctx_s.aggregate(U, out_s)
     boxes_s = final_mailboxes(ctx_s)
-    for variant in (0, 4000, 6, 2):
+    for variant in (0, 6, 2, 1005):
         ctx = B.Brace(n, 0, d, B.default_params(lam=lam, zero_sign=zs, agg_mode=B.AGG_FUSED))
         ctx.workspace.fill_(0x33)
         ctx.set_tuning(variant, 0)
