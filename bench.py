@@ -46,8 +46,8 @@ ALL_WORKLOADS = ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5")
 # launch moves this many bytes per element times n * d (traffic grows with n * d: every element is
 # read once).  None where the kernel has changed since its counters were taken.
 TRAFFIC_BYTES_PER_ELEMENT: dict = {
-    ("cfg4", "aggregate"): None,
-    ("cfg4", "inject"): None,
+    ("cfg4", "aggregate"): 4.0196,   # fused_sign_kernel<int8,1,8,256> 1.60003 GB read + 7.27 MB written, ag_all_bits_kernel 0.53 MB
+    ("cfg4", "inject"): 3.8583,      # inject_stats_reg_kernel<80,3,strided> 1.28007 GB read + 263.2 MB written (rest still in L2)
 }
 
 
