@@ -321,7 +321,9 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
  * 1, 2 or 4 float4 per thread (default: 4, fewer for short sub-vectors); adding
  * 100, 200 or 400 picks the staged statistics kernel with 1, 2 or 4 floats per
  * thread, 800 makes the register-resident statistics kernel address rows through
- * its offset table even when they are consecutive.  On large problems
+ * its offset table even when they are consecutive, 900 makes attack 5 with
+ * generated draws compute its normals block by block instead of for a compacted
+ * list of the coordinate pairs that need one.  On large problems
  * (n*d >= 2^27) the fused kernel writes each sub-vector's bits to its owner's row
  * and one share-only launch spreads them to the other rows; adding 1000 forces
  * that at any size, adding 2000 makes the fused kernel write all n rows itself.

@@ -60,7 +60,8 @@ struct brace_ctx {
   int step_vpt = 0;
   int spread_mode = 0;   // 0/1 = owner row + share-only launch when the layout allows, 2 = fused kernel writes all rows
   int stats_vw = 0;
-  int stats_table = 0;   // 1 = statistics kernel addresses rows through the offset table even when they are consecutive
+  int stats_table = 0;
+  int gen_simple = 0;    // 1 = kind 5 with generated draws runs the plain kernel (no compaction of the normals)   // 1 = statistics kernel addresses rows through the offset table even when they are consecutive
 };
 
 namespace {
@@ -446,6 +447,15 @@ int inject_impl(brace_ctx* ctx, const brace_attack* atk, const float* H, int64_t
   int rc = stage_ids(ctx, atk->h_byz_ids, st);
   if (rc != BRACE_OK) return rc;
   const bool rows16 = (ld_h % 4 == 0) && (ld_u % 4 == 0) && aligned16(H) && aligned16(Uo);
+  if (generated && kind == BRACE_ATTACK_SPARSE_NOISE && atk->prob < 0.5f && ctx->gen_simple == 0) {
+    // uniform < prob  <=>  its 24-bit numerator < ceil(prob * 2^24) (the product is exact in float32)
+    const float scaled = std::ceil(atk->prob * 16777216.0f);
+    const uint32_t thr = scaled <= 0.0f ? 0u : (uint32_t)scaled;   // NaN and negatives: nothing passes
+    dim3 grid(tiles((ctx->d + 7) / 8, kThreads), (unsigned)ctx->f);
+    inject_sparse_generated_kernel<<<grid, kThreads, 0, st>>>(ctx->d_ids, Uo, ld_u, ctx->d, atk->seed, atk->round,
+                                                             atk->sigma, thr, (ld_u % 4 == 0 && aligned16(Uo)) ? 1 : 0);
+    return check_launch(ctx);
+  }
   if (generated) {
     dim3 grid(tiles((ctx->d + 3) / 4, kThreads), (unsigned)ctx->f);
     inject_generated_kernel<<<grid, kThreads, 0, st>>>(kind, ctx->d_ids, Uo, ld_u, ctx->d, atk->seed, atk->round,
@@ -719,13 +729,14 @@ int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid) 
   const int step_code = (fused_variant / 10) % 10;   // tens digit: float4 per thread of the hop kernel
   fused_variant %= 10;
   if (fused_variant > 6 || (step_code != 0 && step_code != 1 && step_code != 2 && step_code != 4) ||
-      (stats_code != 0 && stats_code != 1 && stats_code != 2 && stats_code != 4 && stats_code != 8))
+      (stats_code != 0 && stats_code != 1 && stats_code != 2 && stats_code != 4 && stats_code != 8 && stats_code != 9))
     return BRACE_ERR_INVALID_ARG;
   if (spread_code < 0 || spread_code > 2) return BRACE_ERR_INVALID_ARG;
   ctx->spread_mode = spread_code;
   ctx->step_vpt = step_code;
-  ctx->stats_vw = stats_code == 8 ? 0 : stats_code;
+  ctx->stats_vw = (stats_code == 8 || stats_code == 9) ? 0 : stats_code;
   ctx->stats_table = stats_code == 8 ? 1 : 0;
+  ctx->gen_simple = stats_code == 9 ? 1 : 0;
   ctx->fused_variant = fused_variant;
   ctx->fused_grid = fused_grid;
   return BRACE_OK;

@@ -834,6 +834,75 @@ inject_generated_kernel(int kind, const int* __restrict__ ids, float* __restrict
   }
 }
 
+// Kind 5 with the draws made here, for the usual case of a small prob: only the
+// coordinates whose uniform passes the test need a normal, and the Box-Muller
+// transform (log, square root, sine, cosine) costs several times what the
+// uniform does.  A thread owns 8 coordinates (two uniform blocks).  The warp
+// then compacts the coordinate pairs that need a normal into a list in shared
+// memory (ballots give every pair its slot), works the list off 32 pairs at a
+// time with all lanes busy -- the lane that handles a pair draws the pair's
+// block of the normal stream and runs Box-Muller once -- and hands the values
+// back through shared memory to the owners, which store two float4 each.
+// Values and positions are those of inject_generated_kernel.  blockDim.x = 256;
+// grid = (blocks of 2048 coordinates, f Byzantine rows).
+__global__ void __launch_bounds__(256)
+inject_sparse_generated_kernel(const int* __restrict__ ids, float* __restrict__ Uo, int64_t ld_u, int64_t d,
+                               uint64_t seed, uint32_t round, float sigma, uint32_t thr, int vec) {
+  __shared__ uint8_t sm_list[8][128];                // per warp: pairs that need a normal (lane * 4 + pair)
+  __shared__ float2 sm_z[8][128];                    // per warp: the normals of those pairs
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // this thread owns coordinates 8t .. 8t+7
+  const int64_t warp_t0 = t - lane;
+  const uint32_t id = (uint32_t)ids[blockIdx.y];
+  // uniforms: take[e] <=> (word >> 8) * 2^-24 < prob <=> (word >> 8) < thr, thr = ceil(prob * 2^24)
+  uint32_t take = 0;
+  if (t * 8 < d) {
+    const uint4 w0 = draw_block(seed, round, id, kStreamUniform, 2 * t);
+    const uint4 w1 = draw_block(seed, round, id, kStreamUniform, 2 * t + 1);
+    take = (uint32_t)((w0.x >> 8) < thr) | (uint32_t)((w0.y >> 8) < thr) << 1 | (uint32_t)((w0.z >> 8) < thr) << 2 |
+           (uint32_t)((w0.w >> 8) < thr) << 3 | (uint32_t)((w1.x >> 8) < thr) << 4 | (uint32_t)((w1.y >> 8) < thr) << 5 |
+           (uint32_t)((w1.z >> 8) < thr) << 6 | (uint32_t)((w1.w >> 8) < thr) << 7;
+  }
+  // compaction: pair p of this lane gets slot (pairs of slots < p in the warp) + (lower lanes' pairs of slot p)
+  int total = 0;
+#pragma unroll
+  for (int p = 0; p < 4; ++p) {
+    const bool need = (take >> (2 * p)) & 3u;
+    const uint32_t m = __ballot_sync(0xffffffffu, need);
+    if (need) sm_list[warp][total + __popc(m & ((1u << lane) - 1u))] = (uint8_t)(lane * 4 + p);
+    total += __popc(m);
+  }
+  __syncwarp();
+  for (int i = lane; i < total; i += 32) {
+    const int pid = sm_list[warp][i];
+    const int owner = pid >> 2, p = pid & 3;
+    // pair p of the owner covers coordinates 8 * (warp_t0 + owner) + 2p, +1: block 2 * (..) + p / 2 of the normal stream
+    const uint4 w = draw_block(seed, round, id, kStreamNormal, 2 * (warp_t0 + owner) + (p >> 1));
+    float z0, z1;
+    if (p & 1) normal_pair(w.z, w.w, z0, z1);
+    else normal_pair(w.x, w.y, z0, z1);
+    sm_z[warp][pid] = make_float2(z0, z1);
+  }
+  __syncwarp();
+  if (t * 8 >= d) return;
+  float v[8];
+#pragma unroll
+  for (int p = 0; p < 4; ++p) {
+    float2 z = make_float2(0.f, 0.f);
+    if ((take >> (2 * p)) & 3u) z = sm_z[warp][lane * 4 + p];
+    v[2 * p] = ((take >> (2 * p)) & 1u) ? __fmul_rn(sigma, z.x) : 0.0f;
+    v[2 * p + 1] = ((take >> (2 * p + 1)) & 1u) ? __fmul_rn(sigma, z.y) : 0.0f;
+  }
+  const int64_t k = t * 8;
+  float* dst = Uo + (int64_t)id * ld_u + k;
+  if (vec && k + 8 <= d) {
+    __stcs(reinterpret_cast<float4*>(dst), make_float4(v[0], v[1], v[2], v[3]));
+    __stcs(reinterpret_cast<float4*>(dst) + 1, make_float4(v[4], v[5], v[6], v[7]));
+  } else {
+    for (int e = 0; e < 8 && k + e < d; ++e) dst[e] = v[e];
+  }
+}
+
 // 128-bit variant of the element-wise alterations (rows 16-byte aligned).
 __global__ void __launch_bounds__(256)
 inject_elementwise_vec_kernel(int kind, const int* __restrict__ ids, const float* H, int64_t ld_h, float* Uo,

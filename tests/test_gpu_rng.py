@@ -123,6 +123,34 @@ def test_attacks_with_generated_draws(name, d, ld, ids):
     ctx.close()
 
 
+@pytest.mark.parametrize("d,ld", [(1_000_003, 1_000_064), (65_537, 65_539), (7, 8), (2048, 2048)])
+@pytest.mark.parametrize("prob", [0.1, 0.0, 0.4999, 1e-4])
+def test_sparse_noise_kernels_agree(d, ld, prob):
+    """Attack 5 drawing in the kernel has two forms (normals computed for every block that needs one, or
+    only for the compacted list of coordinate pairs that need one): same bits, at any prob and tail."""
+    n, f = 5, 3
+    H = torch.zeros((n, ld), dtype=torch.float32, device="cuda")
+    rows = []
+    for code in (0, 900):
+        ctx = B.Brace(n, f, d)
+        ctx.set_tuning(code, 0)
+        U = torch.full_like(H, 3.0)
+        ctx.inject_attack(B.make_attack(B.ATTACK_SPARSE_NOISE, sigma=2.5, prob=prob, byz_ids=[4, 0, 2], seed=31337,
+                                        round_idx=9), H, U)
+        rows.append(U)
+        ctx.close()
+    assert torch.equal(rows[0].view(torch.int32), rows[1].view(torch.int32))
+    assert torch.equal(rows[0][[1, 3]], torch.full_like(H, 3.0)[[1, 3]])             # honest rows untouched
+    assert (rows[0][:, d:] == 3.0).all()                                             # padding untouched
+    frac = float((rows[0][[0, 2, 4], :d] != 0).float().mean())
+    assert abs(frac - prob) < 0.02 + 3.0 / d ** 0.5
+    if d <= 70_000:
+        noise, unif = O.attack_draws(O.ATTACK_SPARSE_NOISE, 31337, 9, [4, 0, 2], d)
+        exp = O.inject_attack(O.ATTACK_SPARSE_NOISE, np.zeros((n, d), np.float32), [4, 0, 2], sigma=2.5, prob=prob,
+                              noise=noise, uniform=unif)
+        assert_close_normals(rows[0].cpu().numpy()[[4, 0, 2], :d], exp[[4, 0, 2]])
+
+
 def test_generated_draws_change_with_round_and_seed_and_bad_round_is_refused():
     w = W.scaled(W.WORKLOADS["cfg2"], 4_096)
     H = W.honest_updates(w, 0, device="cuda")
