@@ -788,25 +788,27 @@ int brace_apply_update(brace_ctx* ctx, const void* d_out, int64_t out_ld, float*
   if (!d_weights || ld_weights < ctx->d || !std::isfinite(eta)) return BRACE_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(d_weights) & 3u) != 0) return BRACE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  dim3 grid(tiles(ctx->d, kThreads * 4), (unsigned)ctx->n);
   const bool wvec = (ld_weights % 4 == 0) && aligned16(d_weights);
+  constexpr int kUpt = 4;                            // float4 per thread on the aligned path
+  dim3 grid_v(tiles(ctx->d, kThreads * 4 * kUpt), (unsigned)ctx->n);
+  dim3 grid_s(tiles(ctx->d, kThreads * 4), (unsigned)ctx->n);
   if (ctx->p.rule == BRACE_RULE_SUM) {
     // the rows hold the sum (or already the mean): w <- w - (eta/n) * sum, or w - eta * mean
     const float scale = ctx->p.mean ? eta : eta / (float)ctx->n;
     const bool vec = wvec && (out_ld % 4 == 0) && aligned16(d_out);
     if (vec)
-      apply_update_f32_kernel<true><<<grid, kThreads, 0, st>>>((const float*)d_out, out_ld, d_weights, ld_weights,
-                                                              ctx->d, scale);
+      apply_update_f32_kernel<true, kUpt><<<grid_v, kThreads, 0, st>>>((const float*)d_out, out_ld, d_weights,
+                                                                      ld_weights, ctx->d, scale);
     else
-      apply_update_f32_kernel<false><<<grid, kThreads, 0, st>>>((const float*)d_out, out_ld, d_weights, ld_weights,
-                                                               ctx->d, scale);
+      apply_update_f32_kernel<false, 1><<<grid_s, kThreads, 0, st>>>((const float*)d_out, out_ld, d_weights,
+                                                                    ld_weights, ctx->d, scale);
   } else {
     if (wvec)
-      apply_update_bits_kernel<true><<<grid, kThreads, 0, st>>>((const uint32_t*)d_out, out_ld, d_weights,
-                                                               ld_weights, ctx->d, eta);
+      apply_update_bits_kernel<true, kUpt><<<grid_v, kThreads, 0, st>>>((const uint32_t*)d_out, out_ld, d_weights,
+                                                                       ld_weights, ctx->d, eta);
     else
-      apply_update_bits_kernel<false><<<grid, kThreads, 0, st>>>((const uint32_t*)d_out, out_ld, d_weights,
-                                                                ld_weights, ctx->d, eta);
+      apply_update_bits_kernel<false, 1><<<grid_s, kThreads, 0, st>>>((const uint32_t*)d_out, out_ld, d_weights,
+                                                                     ld_weights, ctx->d, eta);
   }
   return check_launch(ctx);
 }

@@ -597,46 +597,75 @@ fused_sum_kernel(const FusedArgs a) {
 // plain ring-all-reduce (Section 2.2): w <- w - scale*sum with scale = eta/n.
 // grid = (tiles over d, n clients); 4 coordinates per thread.
 // ---------------------------------------------------------------------------
-template <bool VEC>
+// VEC: 16-byte aligned rows; a thread then handles UPT float4 (one output word's worth of
+// coordinates is 8 float4), all loaded before any is stored.
+template <bool VEC, int UPT>
 __global__ void __launch_bounds__(256)
 apply_update_bits_kernel(const uint32_t* __restrict__ out, int64_t out_ld, float* __restrict__ Wt, int64_t ld_w,
                          int64_t d, float eta) {
   const int c = blockIdx.y;
-  const int64_t k = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-  if (k >= d) return;
-  const uint32_t nib = (__ldg(out + (int64_t)c * out_ld + (k >> 5)) >> (int)(k & 31)) & 0xFu;
-  float* w = Wt + (int64_t)c * ld_w + k;
-  if (VEC && k + 4 <= d) {
-    float4 v = *reinterpret_cast<float4*>(w);
-    v.x = __fsub_rn(v.x, (nib & 1u) ? eta : -eta);
-    v.y = __fsub_rn(v.y, (nib & 2u) ? eta : -eta);
-    v.z = __fsub_rn(v.z, (nib & 4u) ? eta : -eta);
-    v.w = __fsub_rn(v.w, (nib & 8u) ? eta : -eta);
-    *reinterpret_cast<float4*>(w) = v;
-  } else {
-    for (int q = 0; q < 4 && k + q < d; ++q) w[q] = __fsub_rn(w[q], ((nib >> q) & 1u) ? eta : -eta);
+  const int64_t k0 = ((int64_t)blockIdx.x * blockDim.x * UPT + threadIdx.x) * 4;
+  float* wrow = Wt + (int64_t)c * ld_w;
+  const uint32_t* orow = out + (int64_t)c * out_ld;
+  float4 v[UPT];
+  uint32_t nib[UPT];
+#pragma unroll
+  for (int u = 0; u < UPT; ++u) {
+    const int64_t k = k0 + (int64_t)u * blockDim.x * 4;
+    if (k < d) {
+      nib[u] = (__ldg(orow + (k >> 5)) >> (int)(k & 31)) & 0xFu;
+      if (VEC && k + 4 <= d) v[u] = *reinterpret_cast<float4*>(wrow + k);
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < UPT; ++u) {
+    const int64_t k = k0 + (int64_t)u * blockDim.x * 4;
+    if (k >= d) continue;
+    float* w = wrow + k;
+    if (VEC && k + 4 <= d) {
+      v[u].x = __fsub_rn(v[u].x, (nib[u] & 1u) ? eta : -eta);
+      v[u].y = __fsub_rn(v[u].y, (nib[u] & 2u) ? eta : -eta);
+      v[u].z = __fsub_rn(v[u].z, (nib[u] & 4u) ? eta : -eta);
+      v[u].w = __fsub_rn(v[u].w, (nib[u] & 8u) ? eta : -eta);
+      *reinterpret_cast<float4*>(w) = v[u];
+    } else {
+      for (int q = 0; q < 4 && k + q < d; ++q) w[q] = __fsub_rn(w[q], ((nib[u] >> q) & 1u) ? eta : -eta);
+    }
   }
 }
 
-template <bool VEC>
+template <bool VEC, int UPT>
 __global__ void __launch_bounds__(256)
 apply_update_f32_kernel(const float* __restrict__ out, int64_t out_ld, float* __restrict__ Wt, int64_t ld_w,
                         int64_t d, float scale) {
   const int c = blockIdx.y;
-  const int64_t k = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-  if (k >= d) return;
-  const float* g = out + (int64_t)c * out_ld + k;
-  float* w = Wt + (int64_t)c * ld_w + k;
-  if (VEC && k + 4 <= d) {
-    const float4 a = ld_stream(g);
-    float4 v = *reinterpret_cast<float4*>(w);
-    v.x = __fsub_rn(v.x, __fmul_rn(scale, a.x));
-    v.y = __fsub_rn(v.y, __fmul_rn(scale, a.y));
-    v.z = __fsub_rn(v.z, __fmul_rn(scale, a.z));
-    v.w = __fsub_rn(v.w, __fmul_rn(scale, a.w));
-    *reinterpret_cast<float4*>(w) = v;
-  } else {
-    for (int q = 0; q < 4 && k + q < d; ++q) w[q] = __fsub_rn(w[q], __fmul_rn(scale, g[q]));
+  const int64_t k0 = ((int64_t)blockIdx.x * blockDim.x * UPT + threadIdx.x) * 4;
+  float* wrow = Wt + (int64_t)c * ld_w;
+  const float* grow = out + (int64_t)c * out_ld;
+  float4 v[UPT], a[UPT];
+#pragma unroll
+  for (int u = 0; u < UPT; ++u) {
+    const int64_t k = k0 + (int64_t)u * blockDim.x * 4;
+    if (VEC && k + 4 <= d) {
+      a[u] = ld_stream(grow + k);
+      v[u] = *reinterpret_cast<float4*>(wrow + k);
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < UPT; ++u) {
+    const int64_t k = k0 + (int64_t)u * blockDim.x * 4;
+    if (k >= d) continue;
+    float* w = wrow + k;
+    if (VEC && k + 4 <= d) {
+      v[u].x = __fsub_rn(v[u].x, __fmul_rn(scale, a[u].x));
+      v[u].y = __fsub_rn(v[u].y, __fmul_rn(scale, a[u].y));
+      v[u].z = __fsub_rn(v[u].z, __fmul_rn(scale, a[u].z));
+      v[u].w = __fsub_rn(v[u].w, __fmul_rn(scale, a[u].w));
+      *reinterpret_cast<float4*>(w) = v[u];
+    } else {
+      const float* g = grow + k;
+      for (int q = 0; q < 4 && k + q < d; ++q) w[q] = __fsub_rn(w[q], __fmul_rn(scale, g[q]));
+    }
   }
 }
 

@@ -567,6 +567,46 @@ def test_fused_round_medium_sizes(n, d, zs):
     ctx_s.close()
 
 
+def test_inject_inside_stream_capture():
+    """The Byzantine id list is uploaded by the first call that sees it.  That upload must not be recorded
+    into a graph (later eager calls would skip it): a capturing call with a new list is refused, and after
+    one eager call the same list captures and replays fine."""
+    w = W.scaled(W.WORKLOADS["cfg3"], 20_000)
+    H = W.honest_updates(w, 0, device="cuda")
+    byz = [7, 3, 41, 20, 11, 0, 49, 30, 5, 17]
+    atk = B.make_attack(w.attack, scale=w.scale, byz_ids=byz)
+    ctx = B.Brace(w.n, w.f, w.d, B.default_params(lam=w.lam))
+    U, out = H.clone(), ctx.new_output()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        status = B.lib().brace_inject_attack(ctx._ctx, atk, H.data_ptr(), H.stride(0), U.data_ptr(), U.stride(0),
+                                             torch.cuda.current_stream().cuda_stream)
+        out.fill_(0)                                     # the graph must not be empty
+    assert status == B.ERR_UNSUPPORTED
+    assert torch.equal(U, H)
+    ctx.inject_attack(atk, H, U)                         # eager: uploads the list
+    ctx.aggregate(U, out)
+    torch.cuda.synchronize()
+    exp_u, exp_out = U.clone(), out.clone()
+    exp = O.inject_attack(w.attack, H.cpu().numpy()[:, :w.d], byz, scale=w.scale)
+    assert np.array_equal(exp_u.cpu().numpy()[:, :w.d].view(np.uint32), exp.view(np.uint32))
+    U.copy_(H)
+    out.fill_(0)
+    graph2 = torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(graph2, stream=side):
+        ctx.inject_attack(atk, H, U)
+        ctx.aggregate(U, out)
+    U.copy_(H)
+    out.fill_(0)
+    graph2.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(U, exp_u) and torch.equal(out, exp_out)
+    ctx.close()
+
+
 # ------------------------------------------------------------------ attack injection + whole pipeline
 def _np(t):
     return None if t is None else t.cpu().numpy()
