@@ -450,6 +450,9 @@ def measure_workload(B, w, args, device, stream, world, rank, sampler):
     res["gpu_launches_per_step"] = launches_per_round * rounds
     res["roofline_round"] = roof(agg_kernel, agg_alg, res["round_ms"], "aggregate")
     res["roofline_inject"] = roof(inj_kernel, inj_alg, res["inject_ms"], "inject")
+    if generated:
+        res["roofline_inject"]["note"] = ("arithmetic-bound, not HBM-bound: the kernel draws its random numbers "
+                                          "(Philox4x32-10, Box-Muller) and only writes the Byzantine rows")
     res["frac_of_nominal_8tbs"] = {"round": res["roofline_round"]["achieved"] / 8000.0,
                                    "inject": res["roofline_inject"]["achieved"] / 8000.0}
 
