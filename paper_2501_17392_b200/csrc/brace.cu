@@ -299,10 +299,10 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
   a.lam_lo = ctx->lam_lo;
   a.zs = ctx->p.zero_sign;
   a.mean = ctx->p.mean;
-  // sign rules with 16-byte aligned output rows: the kernel writes each sub-vector's bits to its owner's
-  // row and one share-only launch spreads them (long bursts per row instead of 128-byte pieces)
-  // (worth a second launch only on large problems)
-  const bool spread = ctx->p.rule != BRACE_RULE_SUM && (out_ld % 4 == 0) && aligned16(out) && ctx->spread_mode != 2 &&
+  // with 16-byte aligned output rows: the kernel writes each sub-vector's result to its owner's row and one
+  // share-only launch spreads it (long bursts per row instead of one tile's piece per row); worth a second
+  // launch only on large problems
+  const bool spread = (out_ld % 4 == 0) && aligned16(out) && ctx->spread_mode != 2 &&
                       (ctx->spread_mode == 1 || (int64_t)ctx->n * ctx->d >= (int64_t)1 << 27);
   a.owner_only = spread ? 1 : 0;
   const bool zs = ctx->p.zero_sign != 0;
@@ -355,10 +355,15 @@ int launch_fused(brace_ctx* ctx, const float* U, int64_t ld, void* out, int64_t 
   int rc = check_launch(ctx);
   if (rc != BRACE_OK || !spread) return rc;
   const int rows_per_group = 8;
-  dim3 grid(tiles(ctx->seg_max / 128 + 2, kThreads), (unsigned)ctx->n,
-            (unsigned)((ctx->n + rows_per_group - 1) / rows_per_group));
-  const cudaError_t perr =
-      launch_pdl(ag_all_bits_kernel, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, rows_per_group);
+  const unsigned groups = (unsigned)((ctx->n + rows_per_group - 1) / rows_per_group);
+  cudaError_t perr;
+  if (ctx->p.rule == BRACE_RULE_SUM) {
+    dim3 grid(tiles(ctx->seg_max, kThreads * 4), (unsigned)ctx->n, groups);
+    perr = launch_pdl(ag_all_f32_kernel, grid, dim3(kThreads), st, ctx->pt, (float*)out, out_ld, rows_per_group);
+  } else {
+    dim3 grid(tiles(ctx->seg_max / 128 + 2, kThreads), (unsigned)ctx->n, groups);
+    perr = launch_pdl(ag_all_bits_kernel, grid, dim3(kThreads), st, ctx->pt, (uint32_t*)out, out_ld, rows_per_group);
+  }
   return check_launch(ctx, perr);
 }
 

@@ -333,6 +333,36 @@ ag_all_bits_kernel(Part pt, uint32_t* out, int64_t out_ld, int rows_per_group) {
   }
 }
 
+// Share-Only at once for the plain-sum rule: every sub-vector is copied from its owner's row to the
+// n-1 other rows, 4 KB (256 threads x 128 bits) of a sub-vector per CTA and row group.
+// grid = (chunks over the longest sub-vector, n sub-vectors, groups of rows); needs granule % 4 == 0
+// and 16-byte aligned rows.
+__global__ void __launch_bounds__(256)
+ag_all_f32_kernel(Part pt, float* out, int64_t out_ld, int rows_per_group) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int n = pt.n;
+  const int j = blockIdx.y;
+  const int owner = j == 0 ? n - 1 : j - 1;
+  const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+  const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (b + i >= e) return;
+  const int r0 = blockIdx.z * rows_per_group;
+  const int r1 = r0 + rows_per_group < n ? r0 + rows_per_group : n;
+  const float* src = out + (int64_t)owner * out_ld + b + i;
+  if (b + i + 4 <= e) {
+    const float4 v = ld_stream(src);
+    for (int row = r0; row < r1; ++row)
+      if (row != owner) __stcs(reinterpret_cast<float4*>(out + (int64_t)row * out_ld + b + i), v);
+  } else {
+    for (int64_t k = b + i; k < e; ++k) {
+      const float v = out[(int64_t)owner * out_ld + k];
+      for (int row = r0; row < r1; ++row)
+        if (row != owner) out[(int64_t)row * out_ld + k] = v;
+    }
+  }
+}
+
 template <bool VEC>
 __global__ void __launch_bounds__(256)
 ag_step_f32_kernel(Part pt, float* out, int64_t out_ld, int step) {
@@ -577,11 +607,15 @@ fused_sum_kernel(const FusedArgs a) {
         for (int q = 0; q < 4; ++q) acc[v][q] = __fdiv_rn(acc[v][q], fn);
       }
       float* dst = out + b + off[v];
+      // owner_only: client j-1, the owner of sub-vector j, alone gets the result here (Phase III is local
+      // to the owner); a share-only launch copies it to the other rows
+      const int row0 = a.owner_only ? (j == 0 ? n - 1 : j - 1) : 0;
+      const int row1 = a.owner_only ? row0 + 1 : n;
       if (nv[v] == 4) {
         const float4 val = make_float4(acc[v][0], acc[v][1], acc[v][2], acc[v][3]);
-        for (int row = 0; row < n; ++row) *reinterpret_cast<float4*>(dst + (int64_t)row * a.out_ld) = val;
+        for (int row = row0; row < row1; ++row) *reinterpret_cast<float4*>(dst + (int64_t)row * a.out_ld) = val;
       } else {
-        for (int row = 0; row < n; ++row) {
+        for (int row = row0; row < row1; ++row) {
 #pragma unroll
           for (int q = 0; q < 3; ++q)
             if (q < nv[v]) dst[(int64_t)row * a.out_ld + q] = acc[v][q];

@@ -256,8 +256,9 @@ def test_full_size_sum_rule_cfg2():
     w = W.WORKLOADS["cfg2"]
     H = W.honest_updates(w, 0, device="cuda")
     outs = []
-    for mode in (B.AGG_FUSED, B.AGG_STEPWISE):
+    for mode, tuning in ((B.AGG_FUSED, 0), (B.AGG_STEPWISE, 0), (B.AGG_FUSED, 1000)):   # 1000: owner rows + share-only launch
         ctx = B.Brace(w.n, 0, w.d, B.default_params(rule=B.RULE_SUM, agg_mode=mode))
+        ctx.set_tuning(tuning, 0)
         out = ctx.new_output()
         ctx.aggregate(H, out)
         torch.cuda.synchronize()
@@ -265,6 +266,7 @@ def test_full_size_sum_rule_cfg2():
         bounds = [ctx.segment(j) for j in range(w.n)]
         ctx.close()
     assert torch.equal(outs[0][:, :w.d].view(torch.int32), outs[1][:, :w.d].view(torch.int32))
+    assert torch.equal(outs[0][:, :w.d].view(torch.int32), outs[2][:, :w.d].view(torch.int32))
     for c in range(1, w.n):
         assert torch.equal(outs[0][c, :w.d].view(torch.int32), outs[0][0, :w.d].view(torch.int32))
     Hh = H.cpu().numpy()[:, :w.d]
