@@ -330,6 +330,15 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
  * Results do not depend on any of these. */
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid);
 
+/* Debug build only (library compiled with -DBRACE_DEBUG; paper_2501_17392_b200.build.build_debug()): the
+ * ring kernels (the share-reduce, consensus and share-only steps of Section 3 and the fused round) check that
+ * the sub-vector they were handed lies inside the buffers they index and that client indices are in range.
+ * A failed check never traps: it records a code and the CTA skips the sub-vector.  This call waits for the
+ * device, returns the code of the first failed check since the previous call in *h_code (0 = none;
+ * 1 = update row, 2 = mailbox, 3 = output row, 4 = client index) and clears it.  The release build performs no
+ * checks and returns BRACE_ERR_UNSUPPORTED with *h_code = 0.  Errors: INVALID_ARG (null), CUDA. */
+int brace_debug_status(int32_t* h_code);
+
 /* Bytes of mailbox scratch built into the library for brace_aggregate_static. */
 #define BRACE_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
 

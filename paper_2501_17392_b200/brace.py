@@ -13,7 +13,8 @@ import os
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libbrace.so")
+# BRACE_LIBRARY names another build of the same library (the debug build, for instance)
+LIB_PATH = os.environ.get("BRACE_LIBRARY") or os.path.join(_PKG, "libbrace.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BAD_STEP, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
 RULE_SIGN_CONSENSUS, RULE_SUM, RULE_MAJORITY_SIGN, RULE_ABS_CONSENSUS = 0, 1, 2, 3
@@ -79,6 +80,7 @@ SIGNATURES = {
     "brace_debug_mailbox": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_int64),
                                       C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
     "brace_set_tuning": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
+    "brace_debug_status": (C.c_int, [C.POINTER(C.c_int32)]),
     "brace_aggregate_static": (C.c_int, [C.c_int32, C.c_int64, C.POINTER(Params), C.c_void_p, C.c_int64, C.c_void_p,
                                          C.c_int64, C.c_void_p]),
 }
@@ -168,6 +170,13 @@ def draw_matrix(what: int, seed: int, round_idx: int, first_client: int, out: to
     """Fill `out` [rows, ld] with the library's own uniform / normal draws of clients
     first_client .. first_client + rows - 1 (the draws attacks 2 and 5 consume)."""
     _check(draw_matrix_status(what, seed, round_idx, first_client, out, d, mu, sigma, stream), "brace_draw_matrix")
+
+
+def debug_status():
+    """(status, code): code of the first index check that failed in a debug build since the last call."""
+    code = C.c_int32(0)
+    status = lib().brace_debug_status(C.byref(code))
+    return status, code.value
 
 
 def aggregate_static_status(n: int, d: int, params: Params, updates: torch.Tensor, out: torch.Tensor,

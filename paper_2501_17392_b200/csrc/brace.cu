@@ -967,6 +967,25 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
   return BRACE_OK;
 }
 
+int brace_debug_status(int32_t* h_code) {
+  if (!h_code) return BRACE_ERR_INVALID_ARG;
+  *h_code = 0;
+#ifdef BRACE_DEBUG
+  int code = 0;
+  const int zero = 0;
+  cudaError_t err = cudaMemcpyFromSymbol(&code, g_debug_status, sizeof(int));     // waits for the device
+  if (err == cudaSuccess) err = cudaMemcpyToSymbol(g_debug_status, &zero, sizeof(int));
+  if (err != cudaSuccess) {
+    g_last_cuda_no_ctx = (int)err;
+    return BRACE_ERR_CUDA;
+  }
+  *h_code = code;
+  return BRACE_OK;
+#else
+  return BRACE_ERR_UNSUPPORTED;
+#endif
+}
+
 int brace_aggregate_static(int32_t n, int64_t d, const brace_params* params, const float* d_updates, int64_t ld,
                            void* d_out, int64_t out_ld, brace_stream_t stream) {
   if (n < 2 || d < 1 || !params_ok(params)) return BRACE_ERR_INVALID_ARG;

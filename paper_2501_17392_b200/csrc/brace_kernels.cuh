@@ -27,6 +27,23 @@ struct Part {
 
 __device__ __forceinline__ int next_client(int c, int n) { return c + 1 == n ? 0 : c + 1; }
 
+// Debug build (-DBRACE_DEBUG): every ring kernel checks, before it touches memory, that the sub-vector
+// it was handed lies inside the buffers it will index (update rows, mailboxes, output rows) and that
+// its client indices are in range.  A check that fails records its code in a status word the host
+// reads with brace_debug_status, and the CTA skips the sub-vector (the checks are uniform over a CTA, so
+// no barrier is left waiting): nothing traps, the context stays usable.  In the release build every
+// check is the constant true.
+enum { kDbgUpdateRow = 1, kDbgMailbox = 2, kDbgOutputRow = 3, kDbgClient = 4 };
+#ifdef BRACE_DEBUG
+__device__ int g_debug_status = 0;                   // code of the first violation since the last read
+__device__ __forceinline__ bool debug_ok(bool cond, int code) {
+  if (!cond) atomicCAS(&g_debug_status, 0, code);
+  return cond;
+}
+#else
+__device__ __forceinline__ bool debug_ok(bool, int) { return true; }
+#endif
+
 // Section 3 Phase I: element-wise sign.  NaN compares false both ways -> 0.
 template <bool ZS>
 __device__ __forceinline__ int sgn1(float x, int zs) {
@@ -86,6 +103,9 @@ rs_step_sign_kernel(Part pt, const float* __restrict__ U, int64_t ld, const P* _
   if (j < 0) j += n;
   const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
   const int64_t L = e - b;
+  if (!(debug_ok(b >= 0 && b <= e && e <= pt.d && pt.d <= ld, kDbgUpdateRow) && debug_ok(L <= seg_pad, kDbgMailbox) &&
+        debug_ok(r >= 0 && r < n && j >= 0 && j < n, kDbgClient)))
+    return;
   const float* uc = U + (int64_t)c * ld + b;
   const float* ur = U + (int64_t)r * ld + b;
   const P* in = mail_in + (int64_t)c * seg_pad;
@@ -157,6 +177,9 @@ rs_step_sum_kernel(Part pt, const float* __restrict__ U, int64_t ld, const float
   if (j < 0) j += n;
   const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
   const int64_t L = e - b;
+  if (!(debug_ok(b >= 0 && b <= e && e <= pt.d && pt.d <= ld, kDbgUpdateRow) && debug_ok(L <= seg_pad, kDbgMailbox) &&
+        debug_ok(r >= 0 && r < n && j >= 0 && j < n, kDbgClient)))
+    return;
   const float* uc = U + (int64_t)c * ld + b;
   const float* ur = U + (int64_t)r * ld + b;
   const float* in = (step == 0) ? uc : mail_in + (int64_t)c * seg_pad;
@@ -202,6 +225,7 @@ consensus_sign_kernel(Part pt, const P* __restrict__ mail, int64_t seg_pad, uint
   const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
   if (b >= e) return;
   const int64_t w0 = b >> 5, w1 = (e + 31) >> 5;
+  if (!(debug_ok(e - b <= seg_pad && e <= pt.d, kDbgMailbox) && debug_ok(w1 <= out_ld, kDbgOutputRow))) return;
   const int64_t w = w0 + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (w >= w1) return;
   const int64_t k0 = (w << 5) > b ? (w << 5) : b;
@@ -239,6 +263,7 @@ consensus_sum_kernel(Part pt, const float* __restrict__ mail, int64_t seg_pad, f
   const int j = next_client(c, n);
   const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
   const int64_t L = e - b;
+  if (!(debug_ok(L <= seg_pad && b <= e, kDbgMailbox) && debug_ok(e <= pt.d && pt.d <= out_ld, kDbgOutputRow))) return;
   const float* src = mail + (int64_t)c * seg_pad;
   float* dst = out + (int64_t)c * out_ld + b;
   const float fn = (float)n;
@@ -276,6 +301,8 @@ ag_step_bits_kernel(Part pt, uint32_t* out, int64_t out_ld, int step) {
   const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
   if (b >= e) return;
   const int64_t w0 = b >> 5, w1 = (e + 31) >> 5;
+  if (!(debug_ok(w1 <= out_ld && e <= pt.d, kDbgOutputRow) && debug_ok(r >= 0 && r < n && j >= 0 && j < n, kDbgClient)))
+    return;
   const int64_t wt = w0 + ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * WPT;
   if (wt >= w1) return;
   const uint32_t* src = out + (int64_t)c * out_ld;
@@ -315,6 +342,7 @@ ag_all_bits_kernel(Part pt, uint32_t* out, int64_t out_ld, int rows_per_group) {
   const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
   if (b >= e) return;
   const int64_t w0 = b >> 5, w1 = (e + 31) >> 5;
+  if (!(debug_ok(w1 <= out_ld && e <= pt.d, kDbgOutputRow) && debug_ok(owner >= 0 && owner < n, kDbgClient))) return;
   const int64_t wt = w0 + ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (wt >= w1) return;
   const int r0 = blockIdx.z * rows_per_group;
@@ -345,6 +373,8 @@ ag_all_f32_kernel(Part pt, float* out, int64_t out_ld, int rows_per_group) {
   const int j = blockIdx.y;
   const int owner = j == 0 ? n - 1 : j - 1;
   const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
+  if (!(debug_ok(b <= e && e <= pt.d && pt.d <= out_ld, kDbgOutputRow) && debug_ok(owner >= 0 && owner < n, kDbgClient)))
+    return;
   const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (b + i >= e) return;
   const int r0 = blockIdx.z * rows_per_group;
@@ -376,6 +406,7 @@ ag_step_f32_kernel(Part pt, float* out, int64_t out_ld, int step) {
   if (j >= n) j -= n;
   const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
   const int64_t L = e - b;
+  if (!(debug_ok(b <= e && e <= pt.d && pt.d <= out_ld, kDbgOutputRow) && debug_ok(r >= 0 && r < n, kDbgClient))) return;
   const float* src = out + (int64_t)c * out_ld + b;
   float* dst = out + (int64_t)r * out_ld + b;
   const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -439,7 +470,10 @@ fused_sign_kernel(const FusedArgs a) {
     const int64_t b = pt.begin(j), e = (j + 1 == n) ? pt.d : pt.begin(j + 1);
     const int64_t L = e - b;
     const int64_t t0 = (int64_t)k * TILE;
-    if (t0 >= L) continue;                         // uniform over the CTA
+    if (t0 >= L) continue;
+    if (!(debug_ok(b >= 0 && e <= pt.d && pt.d <= a.ld, kDbgUpdateRow) && debug_ok(L <= a.seg_pad, kDbgMailbox) &&
+          debug_ok(j >= 0 && j < n, kDbgClient) && debug_ok(((e + 31) >> 5) <= a.out_ld, kDbgOutputRow)))
+      continue;                                    // uniform over the CTA, like the test above                         // uniform over the CTA
 
     int64_t off[VPT];
     int nv[VPT];
@@ -542,6 +576,9 @@ fused_sum_kernel(const FusedArgs a) {
     const int64_t L = e - b;
     const int64_t t0 = (int64_t)k * TILE;
     if (t0 >= L) continue;
+    if (!(debug_ok(b >= 0 && e <= pt.d && pt.d <= a.ld, kDbgUpdateRow) && debug_ok(L <= a.seg_pad, kDbgMailbox) &&
+          debug_ok(j >= 0 && j < n, kDbgClient) && debug_ok(pt.d <= a.out_ld, kDbgOutputRow)))
+      continue;                                    // uniform over the CTA, like the test above
 
     int64_t off[VPT];
     int nv[VPT];
