@@ -182,15 +182,16 @@ def injection_bytes(w, generated: bool):
     return 4 * (n - f) * d + 4 * f * d, "inject_stats_reg_kernel"
 
 
-def sort_network_pairs(n: int) -> int:
+def sort_network_pairs(n: int, outputs=None) -> int:
     """Compare-exchanges per coordinate of the library's sorting network for n values: Batcher's
     odd-even merge sort for the next power of two, restricted to indices below n rounded up to a
-    multiple of 8 (4 for n <= 4)."""
+    multiple of 8 (4 for n <= 4).  With `outputs` (sorted positions that are read afterwards) only the
+    comparators those positions depend on are counted -- the rest is dead code the compiler removes."""
     nb = 4 if n <= 4 else (n + 7) // 8 * 8
     npow = 1
     while npow < nb:
         npow *= 2
-    pairs, p = 0, 1
+    net, p = [], 1
     while p < npow:
         k = p
         while k >= 1:
@@ -198,10 +199,23 @@ def sort_network_pairs(n: int) -> int:
             for i in range(nb):
                 hi = i + k
                 if i >= first and ((i - first) % (2 * k)) < k and hi < nb and i // (2 * p) == hi // (2 * p):
-                    pairs += 1
+                    net.append((i, hi))
             k //= 2
         p *= 2
-    return pairs
+    if outputs is None:
+        return len(net)
+    live, needed = set(outputs), 0
+    for i, hi in reversed(net):
+        if i in live or hi in live:
+            needed += 1
+            live.update((i, hi))
+    return needed
+
+
+def median_positions(n: int):
+    """Sorted positions the library's median kernel may read for this n (its bucket's candidates)."""
+    nb = 4 if n <= 4 else (n + 7) // 8 * 8
+    return range((nb - 8) // 2 if nb > 8 else 0, min(nb // 2, nb - 1) + 1)
 
 
 def attack_seed(w) -> int:
@@ -592,17 +606,30 @@ def extras_leg(B, w, args, device, stream, live):
         if n <= 128:
             # coordinate-wise median / trimmed mean: arithmetic-bound (sorting network of min/max pairs)
             res = torch.empty(d, dtype=torch.float32, device=device)
-            peaks_now, _ = measured_peaks()
-            alu_peak = 148 * 64 * peaks_now.get("sm_max_mhz", 1965.0) * 1e6
-            pairs = sort_network_pairs(n)
+            # peak: the min/max rate of this GPU, measured now with the library's register-only probe kernel
+            sms = torch.cuda.get_device_properties(device).multi_processor_count
+            probe_out = torch.empty(sms * 8 * 256, dtype=torch.float32, device=device)
+            B.minmax_rate_probe(sms * 8, 2000, probe_out, stream)
+            pa, pb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            rates = []
+            for _ in range(3):
+                pa.record(stream)
+                probe_ops = B.minmax_rate_probe(sms * 8, 20000, probe_out, stream)
+                pb.record(stream)
+                torch.cuda.synchronize()
+                rates.append(probe_ops / (pa.elapsed_time(pb) * 1e-3))
+            alu_peak = float(np.median(rates))
+            del probe_out
             for label, kind, trim in (("median", B.STAT_MEDIAN, 0), ("trimmed_mean", B.STAT_TRIMMED_MEAN, f)):
+                # the median reads a few middle positions only: comparators nothing of that depends on are not run
+                pairs = sort_network_pairs(n, median_positions(n) if kind == B.STAT_MEDIAN else None)
                 ctx.coordinate_stat(kind, trim, U, res, stream)
                 ms = timer.median_ms(lambda: ctx.coordinate_stat(kind, trim, U, res, stream), 3)
                 extras["coordinate_" + label] = {
                     "ms": ms, "elements_per_s": n * d / (ms * 1e-3), "bound": "alu",
                     "compare_exchanges_per_coordinate": pairs, "alu_ops_per_coordinate": 2 * pairs,
                     "achieved_ops_per_s": 2 * pairs * d / (ms * 1e-3), "peak_ops_per_s": alu_peak,
-                    "peak_kind": "derived, not measured: 148 SMs x 64 min/max lanes per clock x max SM clock",
+                    "peak_kind": "measured: min/max operations per second of a register-only probe kernel in this run",
                     "frac": 2 * pairs * d / (ms * 1e-3) / alu_peak, "hbm_gbs": (4 * n * d + 4 * d) / (ms * 1e-3) / 1e9}
             del res
     return extras

@@ -330,6 +330,13 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
  * Results do not depend on any of these. */
 int brace_set_tuning(brace_ctx* ctx, int32_t fused_variant, int32_t fused_grid);
 
+/* Calibration for brace_coordinate_stat's roofline (no counterpart in the paper): launches `blocks` CTAs of
+ * 256 threads that each execute iters * 64 register-to-register min/max operations (the operation the sorting
+ * network of the Section 5.1 baselines is made of) and writes one float per thread to d_out
+ * [blocks * 256].  *ops receives the number of min/max operations the launch performs; time the launch
+ * with events on `stream` to get this GPU's min/max rate.  Errors: INVALID_ARG, CUDA. */
+int brace_minmax_rate_probe(int32_t blocks, int32_t iters, float* d_out, int64_t* ops, brace_stream_t stream);
+
 /* Debug build only (library compiled with -DBRACE_DEBUG; paper_2501_17392_b200.build.build_debug()): the
  * ring kernels (the share-reduce, consensus and share-only steps of Section 3 and the fused round) check that
  * the sub-vector they were handed lies inside the buffers they index and that client indices are in range.

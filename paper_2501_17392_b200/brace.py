@@ -81,6 +81,7 @@ SIGNATURES = {
                                       C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
     "brace_set_tuning": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
     "brace_debug_status": (C.c_int, [C.POINTER(C.c_int32)]),
+    "brace_minmax_rate_probe": (C.c_int, [C.c_int32, C.c_int32, C.c_void_p, C.POINTER(C.c_int64), C.c_void_p]),
     "brace_aggregate_static": (C.c_int, [C.c_int32, C.c_int64, C.POINTER(Params), C.c_void_p, C.c_int64, C.c_void_p,
                                          C.c_int64, C.c_void_p]),
 }
@@ -170,6 +171,14 @@ def draw_matrix(what: int, seed: int, round_idx: int, first_client: int, out: to
     """Fill `out` [rows, ld] with the library's own uniform / normal draws of clients
     first_client .. first_client + rows - 1 (the draws attacks 2 and 5 consume)."""
     _check(draw_matrix_status(what, seed, round_idx, first_client, out, d, mu, sigma, stream), "brace_draw_matrix")
+
+
+def minmax_rate_probe(blocks: int, iters: int, out: torch.Tensor, stream=None) -> int:
+    """Launch the min/max calibration kernel; returns the number of operations it performs."""
+    ops = C.c_int64(0)
+    _check(lib().brace_minmax_rate_probe(blocks, iters, _ptr(out), C.byref(ops), _stream(stream)),
+           "brace_minmax_rate_probe")
+    return ops.value
 
 
 def debug_status():

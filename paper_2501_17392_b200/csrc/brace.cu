@@ -827,10 +827,10 @@ int brace_coordinate_stat(brace_ctx* ctx, int32_t kind, int32_t trim, const floa
   if (kind == BRACE_STAT_TRIMMED_MEAN && (trim < 0 || 2 * (int64_t)trim >= ctx->n)) return BRACE_ERR_INVALID_ARG;
   if (ctx->n > 128) return BRACE_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const unsigned blocks = tiles(ctx->d, 128);
+  const unsigned blocks = tiles(ctx->d, kStatThreads);
   const int n = ctx->n;
 #define BRACE_STAT(NB) \
-  case NB: coordinate_stat_kernel<NB><<<blocks, 128, 0, st>>>(kind, trim, n, d_updates, ld, d_result, ctx->d); break
+  case NB: coordinate_stat_kernel<NB><<<blocks, kStatThreads, 0, st>>>(kind, trim, n, d_updates, ld, d_result, ctx->d); break
   switch (n <= 4 ? 4 : (n + 7) / 8 * 8) {            // n rounded up to a multiple of 8 (4 for the smallest)
     BRACE_STAT(4); BRACE_STAT(8); BRACE_STAT(16); BRACE_STAT(24); BRACE_STAT(32); BRACE_STAT(40); BRACE_STAT(48);
     BRACE_STAT(56); BRACE_STAT(64); BRACE_STAT(72); BRACE_STAT(80); BRACE_STAT(88); BRACE_STAT(96); BRACE_STAT(104);
@@ -965,6 +965,15 @@ int brace_debug_mailbox(const brace_ctx* ctx, int32_t client, int32_t hops_back,
   if (segment) *segment = j;
   if (entry_bytes) *entry_bytes = ctx->entry_bytes;
   return BRACE_OK;
+}
+
+int brace_minmax_rate_probe(int32_t blocks, int32_t iters, float* d_out, int64_t* ops, brace_stream_t stream) {
+  if (blocks < 1 || iters < 1 || !d_out || !ops) return BRACE_ERR_INVALID_ARG;
+  brace_ctx ctx;
+  ctx.no_ctx_call = true;
+  minmax_rate_kernel<<<(unsigned)blocks, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(d_out, iters);
+  *ops = (int64_t)blocks * kThreads * (int64_t)iters * 64;
+  return check_launch(&ctx);
 }
 
 int brace_debug_status(int32_t* h_code) {

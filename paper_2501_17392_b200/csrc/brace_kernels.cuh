@@ -1270,8 +1270,13 @@ __host__ __device__ constexpr int pow2_at_least(int v) {
   return p;
 }
 
+#ifndef BRACE_STAT_TPB
+#define BRACE_STAT_TPB 256
+#endif
+constexpr int kStatThreads = BRACE_STAT_TPB;
+
 template <int NB>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kStatThreads)
 coordinate_stat_kernel(int kind, int trim, int n, const float* __restrict__ U, int64_t ld, float* __restrict__ res,
                        int64_t d) {
   constexpr int NP = pow2_at_least(NB);
@@ -1279,8 +1284,13 @@ coordinate_stat_kernel(int kind, int trim, int n, const float* __restrict__ U, i
   if (kc >= d) return;
   const float* src = U + kc;
   float x[NB];
+  // the host picks NB = n rounded up to a multiple of 8 (4 for n <= 4): only the last 7 (3) slots can be pads
+  constexpr int SURE = NB > 8 ? NB - 7 : 1;
 #pragma unroll
-  for (int i = 0; i < NB; ++i) x[i] = (i < n) ? __ldcs(src + (int64_t)i * ld) : __int_as_float(0x7f800000);
+  for (int i = 0; i < NB; ++i) {
+    if (i < SURE) x[i] = __ldcs(src + (int64_t)i * ld);
+    else x[i] = (i < n) ? __ldcs(src + (int64_t)i * ld) : __int_as_float(0x7f800000);
+  }
   // odd-even merge sort, ascending: merges of runs of length p, comparator distance k
 #pragma unroll
   for (int p = 1; p < NP; p *= 2) {
@@ -1302,8 +1312,9 @@ coordinate_stat_kernel(int kind, int trim, int n, const float* __restrict__ U, i
   if (kind == 0) {                                   // median: middle value, or the mean of the two middle ones
     const int hi_idx = n >> 1, lo_idx = (n - 1) >> 1;
     float vlo = 0.f, vhi = 0.f;
+    // n > NB - 8, so both middle positions lie in [(NB - 8) / 2, NB / 2]
 #pragma unroll
-    for (int i = 0; i < NB; ++i) {
+    for (int i = (NB > 8 ? (NB - 8) / 2 : 0); i <= NB / 2 && i < NB; ++i) {
       if (i == lo_idx) vlo = x[i];
       if (i == hi_idx) vhi = x[i];
     }
@@ -1316,6 +1327,40 @@ coordinate_stat_kernel(int kind, int trim, int n, const float* __restrict__ U, i
     out = __double2float_rn(__ddiv_rn(acc, (double)(n - 2 * trim)));
   }
   res[kc] = out;
+}
+
+// ---------------------------------------------------------------------------
+// Calibration: the rate at which this GPU executes the min/max operations the
+// sorting network is made of, so that coordinate_stat_kernel can be held against
+// a measured peak.  Every thread runs `iters` rounds of four stages of eight
+// independent compare-exchanges on 16 registers (pair distances 1, 2, 4, 8, like
+// the stages of a network): 64 min/max operations per round per thread, no
+// memory traffic but one store at the end.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+minmax_rate_kernel(float* __restrict__ out, int iters) {
+  float x[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) x[i] = (float)((threadIdx.x * 37 + i * 101 + blockIdx.x) % 251);
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int dist = 1; dist < 16; dist <<= 1) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int l = i ^ dist;
+        if (l > i) {
+          const float lo = fminf(x[i], x[l]), hi = fmaxf(x[i], x[l]);
+          x[i] = hi;                                 // descending here, so that no stage finds its pairs in order
+          x[l] = lo;
+        }
+      }
+    }
+    x[0] = -x[0];                                    // keep the data moving between rounds
+  }
+  float acc = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) acc += x[i];
+  out[(int64_t)blockIdx.x * blockDim.x + threadIdx.x] = acc;
 }
 
 }  // namespace brace
