@@ -164,7 +164,9 @@ int brace_destroy(brace_ctx* ctx);
  * equal-sized sub-vectors"; formula at brace_params.granule).  Host only. */
 int brace_segment(const brace_ctx* ctx, int32_t j, int64_t* begin, int64_t* end);
 
-/* cudaError_t of the last failed runtime call on this context (0 if none). */
+/* cudaError_t of the last failed runtime call on this context (0 if none).  With ctx = NULL: of the
+ * last failed runtime call made on the calling host thread by an entry point that takes no context
+ * (brace_aggregate_static, brace_draw_matrix, brace_minmax_rate_probe, brace_debug_status). */
 int brace_last_cuda_error(const brace_ctx* ctx);
 
 /* Threat model of Section 3: Byzantine clients alter their vectors before the
@@ -373,9 +375,13 @@ int brace_debug_status(int32_t* h_code);
  * under the sign rule, d <= 1.0 million under the sum rule); larger requests
  * return BRACE_ERR_WORKSPACE and launch nothing.
  *
- * The first call on each device looks up the array's device address (with that
- * device current); make that first call outside any stream capture.  All calls
- * on a device share the one array: it keeps whatever the previous call left
+ * Every call looks up the array's device address for the device that is current
+ * (cudaGetSymbolAddress: no allocation; nothing is cached, so the call stays
+ * valid after a device reset).  The first call on a device also makes the CUDA
+ * runtime load the library's kernels there: make that first call outside any
+ * stream capture.  A CUDA failure of this call is kept per host thread and
+ * returned by brace_last_cuda_error(NULL).  All calls on a device share the one
+ * array: it keeps whatever the previous call left
  * (nothing in it has to start at zero -- the kernel only writes it), and two
  * calls whose kernels may overlap on the GPU (different streams) race on it:
  * serialise them.  Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */
