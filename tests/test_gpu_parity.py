@@ -567,6 +567,54 @@ def test_fused_round_medium_sizes(n, d, zs):
     ctx_s.close()
 
 
+def test_random_shapes_rules_and_layouts():
+    """Seeded random draws of (n, d, granule, row stride, rule, lambda, zero_sign, mean): the whole round by
+    step calls with every mailbox compared after every hop, then by brace_aggregate in both modes, against
+    the oracle's hop-by-hop trace.  Meant to hit combinations the hand-picked cases do not."""
+    rng = np.random.default_rng(20250117392)
+    rules = [B.RULE_SIGN_CONSENSUS, B.RULE_SUM, B.RULE_MAJORITY_SIGN, B.RULE_ABS_CONSENSUS]
+    for case in range(40):
+        n = int(rng.integers(2, 24))
+        d = int(rng.choice([rng.integers(1, 40), rng.integers(40, 3000), rng.integers(3000, 40_000)]))
+        G = int(rng.choice([1, 3, 4, 32, 100, 128, 256]))
+        ld = d + int(rng.choice([0, 1, 2, 3, 4, 125]))
+        if rng.random() < 0.5:
+            ld = W.round_up(d, 128)
+        rule = int(rng.choice(rules))
+        lam = float(rng.integers(-n - 2, n + 2)) + float(rng.choice([0.0, 0.5]))
+        zs = int(rng.choice([0, 0, 1, -1]))
+        mean = int(rng.random() < 0.5)
+        if rng.random() < 0.5:
+            U = W.small_integer_updates(n, d, seed=case, ld=ld)
+        else:
+            U = W.edge_value_updates(n, d, seed=case, ld=ld)
+            if rule == B.RULE_SUM:                     # NaN != NaN would hide nothing but complicates the compare
+                U = torch.nan_to_num(U, nan=0.25, posinf=3.0, neginf=-3.0)
+        Uh = U.numpy()[:, :d]
+        with np.errstate(all="ignore"):
+            tr = O.ring_round(Uh, rule=rule, lam=lam, zero_sign=zs, granule=G, mean=bool(mean))
+        Ud = U.cuda()
+        tag = (case, n, d, G, ld, rule, lam, zs, mean)
+        ctx = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, zero_sign=zs, granule=G, mean=mean,
+                                                agg_mode=B.AGG_STEPWISE))
+        out = ctx.new_output()
+        run_steps_and_check(ctx, Ud, tr, out, rule, d)
+        check_final(out, tr, rule, d)
+        out.fill_(0)
+        ctx.aggregate(Ud, out)
+        check_final(out, tr, rule, d)
+        ctx.close()
+        ctxa = B.Brace(n, 0, d, B.default_params(rule=rule, lam=lam, zero_sign=zs, granule=G, mean=mean,
+                                                 agg_mode=B.AGG_AUTO))
+        outa = ctxa.new_output()
+        ctxa.aggregate(Ud, outa)
+        try:
+            check_final(outa, tr, rule, d)
+        except AssertionError as exc:
+            raise AssertionError(f"case {tag}: {exc}") from exc
+        ctxa.close()
+
+
 def test_inject_inside_stream_capture():
     """The Byzantine id list is uploaded by the first call that sees it.  That upload must not be recorded
     into a graph (later eager calls would skip it): a capturing call with a new list is refused, and after
