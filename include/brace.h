@@ -265,7 +265,7 @@ int brace_coordinate_stat(brace_ctx* ctx, int32_t kind, int32_t trim, const floa
  * row i of d_out [rows][ld] belongs to client first_client + i;
  *   what = BRACE_DRAW_UNIFORM  d_out[i][k] = the uniform of (seed, round, client, k)
  *   what = BRACE_DRAW_NORMAL   d_out[i][k] = mu + sigma * z, z the normal of (seed, round, client, k)
- * Needs no context.  Errors: INVALID_ARG (null, rows < 1, d < 1, ld < d,
+ * Needs no context.  Errors: INVALID_ARG (null, rows < 1 or > 65535, d < 1, ld < d,
  * first_client < 0, round >= 2^24), CUDA. */
 enum { BRACE_DRAW_UNIFORM = 0, BRACE_DRAW_NORMAL = 1 };
 int brace_draw_matrix(int32_t what, uint64_t seed, uint32_t round, int32_t first_client, int32_t rows, int64_t d,
